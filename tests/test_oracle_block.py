@@ -1,0 +1,296 @@
+"""Pins for the oracle's block math (Eq. 2 with scale/shift), the cache merge (Eq. 3),
+linear extrapolation (Eq. 5) and the step schedule (Algorithm 1).  CPU only.
+
+The block's pieces reduce to library routines (layer_norm, scaled-dot-product
+attention, GELU-tanh, SiLU, linear); each is checked against torch's float64
+implementation, and the cached step is checked against the uncached forward in the
+case where the paper says they coincide (refresh ratio 1, no extrapolation)."""
+import numpy as np
+import pytest
+import torch
+import torch.nn.functional as TF
+
+from oracle import hero_oracle as O
+from workloads import synthetic as S
+
+
+def small_cfg(**kw):
+    base = dict(n_blocks=2, n_shallow=2, hidden=32, n_heads=2, head_dim=16, ffn_dim=64, temb_dim=12,
+                batch=2, frames=2, grid_h=4, grid_w=5, n_text=3, patch_h=2, patch_w=2,
+                ratio_num=1, ratio_den=4, quota_mode=0, seed=11, warmup_full_steps=2, full_interval=0)
+    base.update(kw)
+    return O.Config(**base)
+
+
+def rand_weights(cfg, scale=0.2, seed=0):
+    rng = np.random.default_rng(seed)
+    d = dict(cfg.__dict__, dtype="fp32")
+    return [{k: rng.standard_normal(shp) * scale for k, shp in S.weight_shapes(d).items()}
+            for _ in range(cfg.n_blocks)]
+
+
+def t64(a):
+    return torch.from_numpy(np.asarray(a, np.float64))
+
+
+# ---------------------------------------------------------------- elementary routines
+def test_layernorm_modulate_vs_torch():
+    cfg = small_cfg()
+    rng = np.random.default_rng(0)
+    x, sh, sc = rng.standard_normal((7, 32)) * 3 + 1, rng.standard_normal(32), rng.standard_normal(32)
+    want = TF.layer_norm(t64(x), (32,), eps=1e-5) * (1 + t64(sc)) + t64(sh)
+    np.testing.assert_allclose(O.layernorm_modulate(cfg, x, sh, sc), want.numpy(), rtol=1e-12, atol=1e-12)
+
+
+def test_gelu_and_silu_vs_torch():
+    t = np.linspace(-6, 6, 1001)
+    np.testing.assert_allclose(O.gelu_tanh(t), TF.gelu(t64(t), approximate="tanh").numpy(), rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(O.silu(t), TF.silu(t64(t)).numpy(), rtol=1e-12, atol=1e-13)
+
+
+def test_attention_vs_torch_sdpa_and_rows_sum_to_one():
+    cfg = small_cfg(hidden=48, n_heads=3, head_dim=16)
+    rng = np.random.default_rng(1)
+    n, N = 5, 23
+    q, k, v = rng.standard_normal((n, 48)), rng.standard_normal((N, 48)), rng.standard_normal((N, 48))
+    got = O.attention(cfg, q, k, v)
+    th = lambda a, m: t64(a).reshape(m, 3, 16).transpose(0, 1)      # [heads, m, hd]
+    want = TF.scaled_dot_product_attention(th(q, n), th(k, N), th(v, N)).transpose(0, 1).reshape(n, 48)
+    np.testing.assert_allclose(got, want.numpy(), rtol=1e-11, atol=1e-12)
+    # with V = all ones the output is exactly the sum of the probabilities
+    np.testing.assert_allclose(O.attention(cfg, q, k, np.ones_like(v)), 1.0, rtol=1e-12)
+    # a query is dominated by the key it matches when scaled up
+    big = O.attention(cfg, 200 * k[[4]], k, v)
+    assert np.abs(big - v[4]).max() < 1e-6
+
+
+def test_modulation_split_order():
+    cfg = small_cfg(has_gate=1)
+    w = rand_weights(cfg)[0]
+    temb = np.random.default_rng(2).standard_normal((2, 12))
+    m = (TF.silu(t64(temb)) @ t64(w["w_mod"]).T + t64(w["b_mod"])).numpy()
+    parts = O.modulation(cfg, w, temb)
+    assert len(parts) == 6
+    for i, p in enumerate(parts):                  # shift1, scale1, shift2, scale2, gate1, gate2
+        np.testing.assert_allclose(p, m[:, i * 32:(i + 1) * 32], rtol=1e-12)
+
+
+# ---------------------------------------------------------------- the whole block vs a torch block
+def torch_block(cfg, w, x, temb):
+    D, hd, nh = cfg.hidden, cfg.head_dim, cfg.n_heads
+    w = {k: t64(v) for k, v in w.items()}
+    x, temb = t64(x), t64(temb)
+    m = TF.linear(TF.silu(temb), w["w_mod"], w["b_mod"])
+    ch = m.chunk(6 if cfg.has_gate else 4, dim=-1)
+    B, N, _ = x.shape
+    a = TF.layer_norm(x, (D,), eps=cfg.eps) * (1 + ch[1][:, None]) + ch[0][:, None]
+    q, k, v = TF.linear(a, w["w_qkv"], w["b_qkv"]).chunk(3, dim=-1)
+    sp = lambda t: t.reshape(B, N, nh, hd).transpose(1, 2)
+    o = TF.scaled_dot_product_attention(sp(q), sp(k), sp(v)).transpose(1, 2).reshape(B, N, D)
+    g = TF.linear(o, w["w_o"], w["b_o"])
+    if cfg.has_gate:
+        g = g * ch[4][:, None]
+    x = x + g
+    a = TF.layer_norm(x, (D,), eps=cfg.eps) * (1 + ch[3][:, None]) + ch[2][:, None]
+    g2 = TF.linear(TF.gelu(TF.linear(a, w["w_1"], w["b_1"]), approximate="tanh"), w["w_2"], w["b_2"])
+    if cfg.has_gate:
+        g2 = g2 * ch[5][:, None]
+    return (x + g2).numpy(), g.numpy(), g2.numpy(), k.numpy(), v.numpy()
+
+
+@pytest.mark.parametrize("gate", [0, 1])
+def test_full_block_vs_torch_library_block(gate):
+    cfg = small_cfg(n_blocks=1, n_shallow=1, has_gate=gate)
+    w = rand_weights(cfg, seed=3)
+    rng = np.random.default_rng(4)
+    x, temb = rng.standard_normal((2, cfg.n_rows, 32)), rng.standard_normal((2, 12))
+    orc = O.HeroOracle(cfg, w)
+    got = orc.block_refresh(0, x.copy(), temb, None)
+    want, g, g2, k, v = torch_block(cfg, w[0], x, temb)
+    np.testing.assert_allclose(got, want, rtol=1e-10, atol=1e-11)
+    st = orc.blocks[0]
+    np.testing.assert_allclose(st.g[0], g, rtol=1e-10, atol=1e-11)
+    np.testing.assert_allclose(st.g[1], g2, rtol=1e-10, atol=1e-11)
+    np.testing.assert_allclose(st.k_cache, k, rtol=1e-10, atol=1e-11)
+    np.testing.assert_allclose(st.v_cache, v, rtol=1e-10, atol=1e-11)
+
+
+# ---------------------------------------------------------------- cached == uncached where the paper says so
+def test_ratio_one_without_extrapolation_equals_uncached_step():
+    """R = 1 makes S(z) = z; with text rows included and every block shallow, a cached
+    step is Eq. 2 on all rows, i.e. the uncached forward, on every step."""
+    cfg = small_cfg(n_blocks=3, n_shallow=3, ratio_num=1, ratio_den=1)
+    w = rand_weights(cfg, seed=5)
+    rng = np.random.default_rng(6)
+    orc = O.HeroOracle(cfg, w)
+    for s in range(4):
+        x, temb = rng.standard_normal((2, cfg.n_rows, 32)), rng.standard_normal((2, 12))
+        want = O.uncached_forward(cfg, w, x, temb)
+        if orc.is_full_step(s):
+            got = orc.step(s, x, temb)
+        else:       # refresh every row (text included) through the refresh path
+            got = np.array(x)
+            for l in range(cfg.n_blocks):
+                vid = orc.select(l)
+                assert len(vid) == cfg.n_video
+                orc.block_refresh(l, got, temb, np.arange(cfg.n_rows))
+        np.testing.assert_allclose(got, want, rtol=1e-10, atol=1e-11)
+
+
+def test_uncached_forward_vs_torch_block_stack():
+    cfg = small_cfg(n_blocks=2, n_shallow=2)
+    w = rand_weights(cfg, seed=8)
+    rng = np.random.default_rng(9)
+    x, temb = rng.standard_normal((2, cfg.n_rows, 32)), rng.standard_normal((2, 12))
+    want = x
+    for blk in w:
+        want = torch_block(cfg, blk, want, temb)[0]
+    np.testing.assert_allclose(O.uncached_forward(cfg, w, x, temb), want, rtol=1e-10, atol=1e-11)
+
+
+# ---------------------------------------------------------------- merge (Eq. 3)
+def test_refresh_touches_only_selected_rows_and_reads_the_full_kv_cache():
+    cfg = small_cfg(n_blocks=1, n_shallow=1)
+    w = rand_weights(cfg, seed=10)
+    rng = np.random.default_rng(12)
+    x0, temb0 = rng.standard_normal((2, cfg.n_rows, 32)), rng.standard_normal((2, 12))
+    orc = O.HeroOracle(cfg, w)
+    orc.block_refresh(0, x0.copy(), temb0, None)
+    st = orc.blocks[0]
+    before = [st.k_cache.copy(), st.v_cache.copy(), st.g[0].copy(), st.g[1].copy()]
+    x1, temb1 = rng.standard_normal((2, cfg.n_rows, 32)), rng.standard_normal((2, 12))
+    rows = orc.select(0)
+    keep = np.setdiff1d(np.arange(cfg.n_rows), rows)
+    x_in = x1.copy()
+    out = orc.block_refresh(0, x1, temb1, rows)
+    after = [st.k_cache, st.v_cache, st.g[0], st.g[1]]
+    for b4, af in zip(before, after):
+        assert np.array_equal(b4[:, keep], af[:, keep])            # bit-identical reuse
+        assert not np.array_equal(b4[:, rows], af[:, rows])
+    # residual: every row received both cached-or-fresh branch outputs
+    np.testing.assert_allclose(out, x_in + st.g[0] + st.g[1], rtol=1e-12, atol=1e-12)
+    # selected rows: recompute by hand against the merged K/V cache
+    b, r = 1, rows[2]
+    mod = O.modulation(cfg, orc.w[0], temb1)
+    a = O.layernorm_modulate(cfg, x_in[b, [r]], mod[0][b], mod[1][b])
+    q = (a @ orc.w[0]["w_qkv"].T + orc.w[0]["b_qkv"])[:, :32]
+    g = O.attention(cfg, q, st.k_cache[b], st.v_cache[b]) @ orc.w[0]["w_o"].T + orc.w[0]["b_o"]
+    np.testing.assert_allclose(st.g[0][b, r], g[0], rtol=1e-11, atol=1e-12)
+    # rows_out spot-check mode gives the same values for the rows it computes
+    orc2 = O.HeroOracle(cfg, w)
+    orc2.block_refresh(0, x0.copy(), temb0, None)
+    rows2 = orc2.select(0)
+    assert np.array_equal(rows, rows2)
+    orc2.block_refresh(0, x_in.copy(), temb1, rows, rows_out=rows[1:4])
+    np.testing.assert_allclose(orc2.blocks[0].g[0][:, rows[1:4]], st.g[0][:, rows[1:4]], rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(orc2.blocks[0].g[1][:, rows[1:4]], st.g[1][:, rows[1:4]], rtol=1e-11, atol=1e-12)
+    assert np.array_equal(orc2.blocks[0].k_cache, st.k_cache)
+
+
+# ---------------------------------------------------------------- extrapolation (Eq. 5)
+def test_extrapolation_is_exact_on_features_linear_in_step():
+    rng = np.random.default_rng(13)
+    A, Bm = rng.standard_normal((3, 17, 8)), rng.standard_normal((3, 17, 8))
+    for s_prev, s_last, s in [(0, 1, 2), (0, 1, 5), (1, 6, 7), (1, 6, 10), (6, 11, 13)]:
+        got = O.extrapolate(A + s_prev * Bm, A + s_last * Bm, s - s_last, s_last - s_prev)
+        np.testing.assert_allclose(got, A + s * Bm, rtol=1e-12, atol=1e-12)
+
+
+def test_extrapolation_special_cases():
+    rng = np.random.default_rng(14)
+    g0, g1 = rng.standard_normal((4, 9)), rng.standard_normal((4, 9))
+    assert np.array_equal(O.extrapolate(g0, g1, 0, 3), g1)              # k = 0: plain reuse
+    assert np.array_equal(O.extrapolate(g1, g1, 2, 3), g1)              # Delta = 0: plain reuse
+    np.testing.assert_allclose(O.extrapolate(g0, g1, 1, 1), 2 * g1 - g0)
+    np.testing.assert_allclose(O.extrapolate(g0, g1, 2, 4), 1.5 * g1 - 0.5 * g0)
+
+
+# ---------------------------------------------------------------- schedule and step bookkeeping (Alg. 1)
+def test_schedule():
+    cfg = small_cfg(warmup_full_steps=2, full_interval=5)
+    orc = O.HeroOracle(cfg, rand_weights(cfg))
+    full = [s for s in range(50) if orc.is_full_step(s)]
+    assert full == [0, 1, 6, 11, 16, 21, 26, 31, 36, 41, 46]
+    cfg0 = small_cfg(warmup_full_steps=2, full_interval=0)
+    orc0 = O.HeroOracle(cfg0, rand_weights(cfg0))
+    assert [s for s in range(10) if orc0.is_full_step(s)] == [0, 1]
+    cfg2 = small_cfg(warmup_full_steps=2, full_interval=2)
+    orc2 = O.HeroOracle(cfg2, rand_weights(cfg2))
+    assert [s for s in range(8) if orc2.is_full_step(s)] == [0, 1, 3, 5, 7]
+
+
+def test_cached_step_extrapolates_with_the_real_gap():
+    """Plant histories that are linear in the step index in the deep blocks; a cached
+    step must then add exactly their value at the current step (pins k and d)."""
+    cfg = small_cfg(n_blocks=3, n_shallow=1, warmup_full_steps=2, full_interval=4)
+    w = rand_weights(cfg, seed=15)
+    rng = np.random.default_rng(16)
+    orc = O.HeroOracle(cfg, w)
+    x = rng.standard_normal((2, cfg.n_rows, 32))
+    temb = rng.standard_normal((2, 12))
+    for s in range(6):                       # full steps: 0, 1, 5
+        orc.step(s, x, temb)
+    assert orc.full_steps == [0, 1, 5]
+    shape = (2, cfg.n_rows, 32)
+    A = [[rng.standard_normal(shape) for _ in range(2)] for _ in range(3)]
+    Bm = [[rng.standard_normal(shape) for _ in range(2)] for _ in range(3)]
+    for l in (1, 2):
+        for i in range(2):
+            orc.blocks[l].g_prev[i] = A[l][i] + 1 * Bm[l][i]
+            orc.blocks[l].g_last[i] = A[l][i] + 5 * Bm[l][i]
+    for s in (6, 7, 8):
+        # shallow block 0 runs first; take its output as the deep blocks' input
+        ref = O.HeroOracle(cfg, w)
+        ref.blocks[0] = orc.blocks[0]
+        calls, ages = orc.blocks[0].calls, orc.blocks[0].ages.copy()
+        snapshot = [a.copy() for a in (orc.blocks[0].k_cache, orc.blocks[0].v_cache, *orc.blocks[0].g)]
+        xin = np.array(x)
+        rows = ref.select(0)
+        ref.block_refresh(0, xin, temb, rows)
+        # rewind block 0 and run the real step
+        st = orc.blocks[0]
+        st.calls, st.ages = calls, ages
+        st.k_cache, st.v_cache, st.g[0], st.g[1] = snapshot
+        got = orc.step(s, x, temb)
+        want = xin + sum(A[l][i] + s * Bm[l][i] for l in (1, 2) for i in range(2))
+        np.testing.assert_allclose(got, want, rtol=1e-11, atol=1e-11)
+
+
+def test_history_rotation_and_age_reset_on_full_steps():
+    cfg = small_cfg(n_blocks=2, n_shallow=1, warmup_full_steps=2, full_interval=3)
+    w = rand_weights(cfg, seed=17)
+    rng = np.random.default_rng(18)
+    orc = O.HeroOracle(cfg, w)
+    xs = [rng.standard_normal((2, cfg.n_rows, 32)) for _ in range(5)]
+    te = [rng.standard_normal((2, 12)) for _ in range(5)]
+    orc.step(0, xs[0], te[0])
+    g_step0 = orc.blocks[1].g_last[0].copy()
+    assert orc.blocks[1].g_prev[0] is None
+    orc.step(1, xs[1], te[1])
+    assert np.array_equal(orc.blocks[1].g_prev[0], g_step0)
+    g_step1 = orc.blocks[1].g_last[1].copy()
+    orc.step(2, xs[2], te[2])              # cached
+    assert orc.blocks[0].calls == 1 and orc.blocks[0].ages.max() == 1
+    assert np.array_equal(orc.blocks[1].g_last[1], g_step1)          # untouched by cached steps
+    orc.step(3, xs[3], te[3])              # cached
+    assert orc.blocks[0].calls == 2
+    orc.step(4, xs[4], te[4])              # full (1 + 3)
+    assert orc.full_steps == [0, 1, 4]
+    assert orc.blocks[0].ages.max() == 0 and orc.blocks[0].calls == 2
+    assert np.array_equal(orc.blocks[1].g_prev[1], g_step1)
+
+
+def test_tiny_config_ten_steps_runs_and_follows_schedule():
+    cfgd = S.CONFIGS["tiny"]
+    cfg = O.Config.from_dict(cfgd)
+    w = [S.block_weights(cfgd, l) for l in range(cfg.n_blocks)]
+    orc = O.HeroOracle(cfg, w)
+    x = S.tokens(cfgd)
+    n_sel = []
+    for s in range(cfgd["steps"]):
+        out = orc.step(s, x, S.temb(cfgd, s))
+        assert np.isfinite(out).all()
+    assert orc.full_steps == [0, 1]
+    assert orc.blocks[0].calls == 8 and orc.blocks[1].calls == 8
+    assert orc.blocks[2].calls == 0
+    assert O.n_selected(cfg, 0) == 32           # 25 % of 128 video tokens
