@@ -1,0 +1,169 @@
+/*
+ * hero.h - C ABI of the HERO cached DiT denoising step for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the hot path of "HERO: Hierarchical Extrapolation and
+ * Refresh for Efficient World Models": in shallow blocks a patch-wise,
+ * frequency-aware sampler picks tokens, only those rows are recomputed through
+ * attention and the FFN and merged back into a per-block feature cache (Sec. 4.3,
+ * Eq. 3, Eq. 4); in deep blocks attention and FFN are skipped and the branch
+ * outputs are linearly extrapolated from two cached steps (Sec. 4.4, Eq. 5);
+ * Algorithm 1 sequences the two.
+ *
+ * Conventions
+ *   - Every pointer named d_* is DEVICE memory, h_* is HOST memory.  The caller
+ *     owns all buffers it passes; the context owns every cache, counter and
+ *     workspace it allocates in hero_init and frees them in hero_destroy.
+ *   - Sequence layout: x is [batch, N, hidden] row-major, N = n_text + frames *
+ *     grid_h * grid_w; the n_text text rows come first, then video tokens in
+ *     (frame, y, x) order.  Run dtype (fp32 or bf16) applies to x, temb, weights
+ *     and caches alike.
+ *   - Weight matrices are row-major [out_features, in_features] (K contiguous).
+ *     Device pointers must be 16-byte aligned; in bf16 mode hidden, ffn_dim and
+ *     temb_dim must be multiples of 8 and head_dim must be 64.
+ *   - All work is enqueued on the CUDA stream given to hero_init; no call
+ *     synchronises the device unless stated.  Calls on one context must not
+ *     overlap in time.
+ *   - Return value: HERO_OK (0) or a negative HERO_ERR_* code.  After an argument
+ *     error nothing has been launched.  No exception crosses this boundary.
+ */
+#ifndef HERO_H_
+#define HERO_H_
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define HERO_OK            0
+#define HERO_ERR_ARG      -1   /* NULL pointer, size out of range, inconsistent config */
+#define HERO_ERR_ALIGN    -2   /* pointer not 16-byte aligned / dimension not vectorisable */
+#define HERO_ERR_CAP      -3   /* index list capacity too small */
+#define HERO_ERR_STATE    -4   /* call order violated (e.g. cached step before any full step) */
+#define HERO_ERR_CUDA     -5   /* a CUDA runtime/driver call failed; see hero_last_cuda_error */
+#define HERO_ERR_TIMEOUT  -6   /* a bounded device-side wait ran out (reported by hero_check_status) */
+#define HERO_ERR_NOMEM    -7   /* device allocation failed */
+
+#define HERO_DTYPE_FP32 0
+#define HERO_DTYPE_BF16 1
+
+typedef struct hero_ctx hero_ctx;   /* opaque */
+
+/* Hyper-parameters of Algorithm 1 and the DiT block shape. */
+typedef struct hero_config {
+  int n_blocks;            /* L */
+  int n_shallow;           /* blocks [0, n_shallow) refresh ("l < K"), the rest extrapolate */
+  int hidden, n_heads, head_dim, ffn_dim, temb_dim;
+  int batch, frames, grid_h, grid_w, n_text;
+  int patch_h, patch_w;    /* p_h x p_w spatial patches inside each frame (Sec. 4.3) */
+  int ratio_num, ratio_den;/* refresh ratio R as an exact rational, 0 < R <= 1 */
+  int quota_mode;          /* 0: running-floor split of R*#P; 1: round-half-up(R*#P) */
+  int warmup_full_steps;   /* leading steps that are always full ("initial caching") */
+  int full_interval;       /* M: a full step every M steps after warm-up; 0 = never */
+  int dtype;               /* HERO_DTYPE_* */
+  int has_gate;            /* 1: adaLN also yields a gate per branch (6 chunks instead of 4) */
+  unsigned long long seed; /* low 32 bits seed the sampler's counter-based hash */
+} hero_config;
+
+/* Device pointers to one block's parameters (borrowed for the context's lifetime).
+ * w_mod [n_mod*hidden, temb_dim] with chunks (shift1, scale1, shift2, scale2[, gate1, gate2]);
+ * w_qkv [3*hidden, hidden] with output chunks (q, k, v); w_o [hidden, hidden];
+ * w_1 [ffn_dim, hidden]; w_2 [hidden, ffn_dim]; biases match the output size. */
+typedef struct hero_block_weights {
+  const void *w_mod, *b_mod, *w_qkv, *b_qkv, *w_o, *b_o, *w_1, *b_1, *w_2, *b_2;
+} hero_block_weights;
+
+/* ---- context ------------------------------------------------------------- */
+
+/* Validate cfg, allocate caches (K, V, G_attn, G_ffn per shallow block; two history
+ * slots x two branches per deep block), age counters, workspace and TMA descriptors
+ * on the current device.  blocks[n_blocks] is copied; the weights it points to are
+ * not.  cuda_stream is a cudaStream_t (NULL = legacy default stream). */
+int hero_init(hero_ctx **out, const hero_config *cfg, const hero_block_weights *blocks, void *cuda_stream);
+/* Forget all cached state (ages, call counters, step history); memory is kept. */
+int hero_reset(hero_ctx *ctx);
+void hero_destroy(hero_ctx *ctx);
+const char *hero_strerror(int code);
+/* Synchronise the context's stream and return HERO_ERR_TIMEOUT if any kernel gave up on
+ * a bounded wait since the last check, HERO_ERR_CUDA on a CUDA error, else HERO_OK. */
+int hero_check_status(hero_ctx *ctx);
+/* Text of the last failing CUDA call on this thread ("" if none). */
+const char *hero_last_cuda_error(void);
+/* Bytes of device memory the context allocated. */
+long long hero_device_bytes(const hero_ctx *ctx);
+
+/* ---- the method's calls (Algorithm 1) ------------------------------------ */
+
+/* S(z) of Eq. 4 for one shallow block: per patch take the quota's worth of tokens with the
+ * largest keys (age+1)*(hash+1) (frequency-aware tracking, Sec. 4.3), reset their ages, age
+ * the rest, and write the selected sequence rows in ascending order to d_idx (int32,
+ * capacity cap).  *n_sel (host, may be NULL) receives the list length, which is a closed
+ * form of the config and the block's call counter; the counter advances by one. */
+int hero_select_tokens(hero_ctx *ctx, int block, int *d_idx, int cap, int *n_sel);
+/* Length hero_select_tokens will produce on its next call for this block. */
+int hero_next_n_sel(const hero_ctx *ctx, int block);
+
+/* Eq. 2 on the rows listed in d_idx (ascending sequence rows, shared by the batch), merged
+ * with the block's cache as in Eq. 3, followed by the residual add for ALL rows:
+ * LN+modulate -> QKV -> K,V rows written to the cache -> attention of the refreshed queries
+ * over the full cached K/V -> out-proj rows into G_attn -> x += G_attn -> LN+modulate ->
+ * FFN (GELU-tanh) rows into G_ffn -> x += G_ffn.  d_idx == NULL with n_sel == N is the full
+ * pass ("initial caching"): all rows, ages reset, deep blocks rotate their history slots.
+ * d_x [batch,N,hidden] is updated in place; d_temb is [batch, temb_dim]. */
+int hero_refresh_block(hero_ctx *ctx, int block, void *d_x, const void *d_temb,
+                       const int *d_idx, int n_sel);
+
+/* Eq. 5 for a deep block, both branches, plus the residual add:
+ * x += g_last + (g_last - g_prev) * k/d for the attention and the FFN history. */
+int hero_extrapolate_block(hero_ctx *ctx, int block, void *d_x, int k, int d);
+
+/* One denoising step through all blocks with Algorithm 1's schedule: a full step when
+ * step < warmup_full_steps or (step - (warmup-1)) % M == 0, else select+refresh in shallow
+ * blocks and extrapolation in deep ones with k, d taken from the recorded full steps. */
+int hero_step(hero_ctx *ctx, int step, void *d_x, const void *d_temb);
+/* Same with HOST buffers: copies h_x and h_temb to the device, runs the step, copies x
+ * back into h_x and synchronises the stream.  Pinned host memory overlaps best. */
+int hero_step_host(hero_ctx *ctx, int step, void *h_x, const void *h_temb);
+/* 1 if hero_step would run `step` as a full step. */
+int hero_is_full_step(const hero_ctx *ctx, int step);
+
+/* ---- isolated kernels (stateless; stream = cudaStream_t) ------------------- */
+
+/* Eq. 5 alone: out = g_last + (g_last - g_prev) * k/d over n_elem elements. */
+int hero_extrapolate(const void *d_g_prev, const void *d_g_last, void *d_out, long long n_elem,
+                     int k, int d, int dtype, void *stream);
+/* dst[b, i, :] = src[b, idx[i], :] for b < B, i < n_sel; src is [B,N,D], dst [B,n_sel,D]. */
+int hero_gather_rows(const void *d_src, const int *d_idx, void *d_dst, int B, int N, int n_sel,
+                     int D, int dtype, void *stream);
+/* dst[b, idx[i], :] = src[b, i, :]; other rows of dst are not touched (Eq. 3's merge). */
+int hero_scatter_rows(const void *d_src, const int *d_idx, void *d_dst, int B, int N, int n_sel,
+                      int D, int dtype, void *stream);
+/* C[M,N] = A[M,K] * W[N,K]^T + bias[N] in bf16 with fp32 accumulation on the tensor cores
+ * (act = 1 applies GELU-tanh).  The GEMM of the refresh path, exposed for tests and timing. */
+int hero_gemm_bf16(const void *d_a, const void *d_w, const void *d_bias, void *d_c,
+                   int M, int N, int K, int act, void *stream);
+/* O[b,i,h,:] = softmax_j(Q[b,i,h,:] . K[b,j,h,:] / sqrt(head_dim)) V[b,j,h,:], j over all N
+ * rows; Q,O are [B,n_q,heads*64] bf16, K,V are [B,N,heads*64] bf16.  No score matrix is stored. */
+int hero_attention_bf16(const void *d_q, const void *d_k, const void *d_v, void *d_o,
+                        int B, int n_q, int N, int heads, void *stream);
+
+/* Synchronise `stream` and return HERO_ERR_TIMEOUT if hero_gemm_bf16 / hero_attention_bf16 gave
+ * up on a bounded device-side wait since the last poll, else HERO_OK. */
+int hero_isolated_status(void *stream);
+
+/* ---- state access for tests and checkpoints -------------------------------- */
+#define HERO_STATE_AGES     0   /* u16[n_video] */
+#define HERO_STATE_CALLS    1   /* int32[1] selection call counter */
+#define HERO_STATE_K        2   /* [B,N,D] run dtype (shallow blocks) */
+#define HERO_STATE_V        3
+#define HERO_STATE_G_ATTN   4   /* shallow: feature cache; deep: g_last */
+#define HERO_STATE_G_FFN    5
+#define HERO_STATE_G_ATTN_PREV 6 /* deep blocks: g_prev */
+#define HERO_STATE_G_FFN_PREV  7
+#define HERO_STATE_STEPS    8   /* int32[3]: number of full steps seen, s_prev, s_last (block ignored) */
+/* Copy a piece of per-block state to / from host memory (synchronises the stream). */
+int hero_state_get(hero_ctx *ctx, int block, int what, void *h_out, long long bytes);
+int hero_state_set(hero_ctx *ctx, int block, int what, const void *h_in, long long bytes);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HERO_H_ */

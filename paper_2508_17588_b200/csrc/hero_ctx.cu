@@ -1,0 +1,569 @@
+// Context, bookkeeping and the C ABI of the HERO cached step (Algorithm 1).
+// All device work is enqueued on the context's stream; the host only does schedule
+// arithmetic (which step is full, the selection list length, k and d of Eq. 5).
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+#include <string>
+#include <vector>
+
+#include "hero_internal.h"
+
+namespace hero {
+
+static thread_local std::string g_last_error;
+void set_cuda_error(cudaError_t e, const char* what) {
+  g_last_error = std::string(what) + ": " + cudaGetErrorString(e);
+}
+
+struct BlockMem {
+  void* k = nullptr;          // shallow: K cache [B,N,D]
+  void* v = nullptr;          // shallow: V cache
+  void* g[2] = {nullptr, nullptr};                       // shallow: G_attn, G_ffn
+  void* hist[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};   // deep: [branch][slot]
+  int last_slot = 0;          // deep: slot holding g_last
+  int n_hist = 0;             // deep: full passes recorded (saturates at 2)
+  uint16_t* ages[2] = {nullptr, nullptr};                // shallow: double-buffered age counters
+  int ages_cur = 0;
+  int calls = 0;              // selections made on this block
+};
+
+}  // namespace hero
+
+using namespace hero;
+
+struct hero_ctx {
+  hero_config cfg;
+  cudaStream_t stream = nullptr;
+  int N = 0, n_video = 0, n_mod = 4, idx_cap = 0;
+  size_t esz = 4;
+  long long elems = 0;                   // B*N*D
+  std::vector<hero_block_weights> w;
+  std::vector<BlockMem> blk;
+  void* kv_tmp[2] = {nullptr, nullptr};  // K/V of deep blocks during full passes (never cached)
+  void *ws_a = nullptr, *ws_q = nullptr, *ws_o = nullptr, *ws_u = nullptr;
+  float* mod = nullptr;                  // [B, n_mod*D] adaLN vectors of the current block
+  int* idx_ws = nullptr;                 // [n_shallow, idx_cap] selection lists of the current step
+  int* d_status = nullptr;
+  void *x_stage = nullptr, *temb_stage = nullptr;
+  int n_full = 0, s_prev = 0, s_last = 0;
+  int mode1_n_sel = 0;
+  long long bytes = 0;
+  std::vector<void*> allocs;
+};
+
+namespace {
+
+int dev_alloc(hero_ctx* c, void** p, size_t bytes) {
+  *p = nullptr;
+  if (bytes == 0) bytes = 16;
+  cudaError_t e = cudaMalloc(p, bytes);
+  if (e != cudaSuccess) {
+    set_cuda_error(e, "cudaMalloc");
+    cudaGetLastError();
+    return HERO_ERR_NOMEM;
+  }
+  c->allocs.push_back(*p);
+  c->bytes += (long long)bytes;
+  return HERO_OK;
+}
+
+SelectGeom geom_of(const hero_config& c) {
+  SelectGeom g;
+  g.frames = c.frames; g.grid_h = c.grid_h; g.grid_w = c.grid_w; g.n_text = c.n_text;
+  g.patch_h = c.patch_h; g.patch_w = c.patch_w;
+  g.ratio_num = c.ratio_num; g.ratio_den = c.ratio_den; g.quota_mode = c.quota_mode;
+  g.seed_lo = (uint32_t)(c.seed & 0xFFFFFFFFull);
+  return g;
+}
+
+// Length of the selection list: a closed form in mode 0 (the running-floor quotas telescope),
+// a constant summed once in mode 1.
+int n_sel_for_call(const hero_ctx* c, int call) {
+  const hero_config& g = c->cfg;
+  if (g.quota_mode == 0) {
+    const long long off = (long long)call * g.patch_h * g.patch_w;
+    return (int)(((c->n_video + off) * g.ratio_num) / g.ratio_den - (off * g.ratio_num) / g.ratio_den);
+  }
+  return c->mode1_n_sel;
+}
+
+int mode1_total(const hero_config& g) {
+  long long total = 0;
+  for (int y0 = 0; y0 < g.grid_h; y0 += g.patch_h)
+    for (int x0 = 0; x0 < g.grid_w; x0 += g.patch_w) {
+      const long long n = (long long)(g.grid_h - y0 < g.patch_h ? g.grid_h - y0 : g.patch_h) *
+                          (g.grid_w - x0 < g.patch_w ? g.grid_w - x0 : g.patch_w);
+      long long q = (2 * n * g.ratio_num + g.ratio_den) / (2 * g.ratio_den);
+      total += q < n ? q : n;
+    }
+  return (int)(total * g.frames);
+}
+
+bool is_full(const hero_config& g, int step) {
+  if (step < g.warmup_full_steps) return true;
+  return g.full_interval > 0 && (step - (g.warmup_full_steps - 1)) % g.full_interval == 0;
+}
+
+int run_gemm(hero_ctx* c, const void* a, const void* w, const void* bias, int M, int Nout, int K, const GemmOut& out) {
+  if (c->cfg.dtype == HERO_DTYPE_BF16) return launch_tc_gemm(a, w, bias, M, Nout, K, out, c->d_status, c->stream);
+  return launch_simt_gemm(a, w, bias, M, Nout, K, out, c->cfg.dtype, c->stream);
+}
+
+int run_attention(hero_ctx* c, const void* q, const void* k, const void* v, void* o, int n_q) {
+  const hero_config& g = c->cfg;
+  if (g.dtype == HERO_DTYPE_BF16)
+    return launch_tc_attention(q, k, v, o, g.batch, n_q, c->N, g.n_heads, c->d_status, c->stream);
+  return launch_simt_attention(q, k, v, o, g.batch, n_q, c->N, g.n_heads, g.head_dim, g.dtype, c->stream);
+}
+
+// Eq. 2 on the listed rows + Eq. 3's merge + the residual adds of Algorithm 1.
+int refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, const int* d_idx, int n_sel) {
+  const hero_config& g = c->cfg;
+  const int B = g.batch, N = c->N, D = g.hidden, F = g.ffn_dim;
+  const bool full = d_idx == nullptr;
+  const bool deep = block >= g.n_shallow;
+  BlockMem& bm = c->blk[block];
+  const hero_block_weights& w = c->w[block];
+  const int M = B * n_sel;
+  const int mod_ld = c->n_mod * D;
+
+  void *kdst, *vdst, *ga, *gf;
+  int new_slot = 0;
+  if (deep) {
+    new_slot = bm.n_hist == 0 ? 0 : (bm.last_slot ^ 1);
+    kdst = c->kv_tmp[0]; vdst = c->kv_tmp[1];
+    ga = bm.hist[0][new_slot]; gf = bm.hist[1][new_slot];
+  } else {
+    kdst = bm.k; vdst = bm.v; ga = bm.g[0]; gf = bm.g[1];
+  }
+
+  HERO_TRY(launch_modulation(d_temb, w.w_mod, w.b_mod, c->mod, B, mod_ld, g.temb_dim, g.dtype, c->stream));
+  const float* shift1 = c->mod;
+  const float* scale1 = c->mod + D;
+  const float* shift2 = c->mod + 2 * D;
+  const float* scale2 = c->mod + 3 * D;
+  const float* gate1 = g.has_gate ? c->mod + 4 * D : nullptr;
+  const float* gate2 = g.has_gate ? c->mod + 5 * D : nullptr;
+
+  // attention branch
+  HERO_TRY(launch_gather_ln_modulate(d_x, nullptr, d_idx, shift1, scale1, mod_ld, c->ws_a, B, N, n_sel, D, 1e-5f,
+                                     g.dtype, c->stream));
+  GemmOut o_qkv = {};
+  o_qkv.ptr[0] = c->ws_q; o_qkv.ld[0] = D; o_qkv.scatter[0] = 0;
+  o_qkv.ptr[1] = kdst;    o_qkv.ld[1] = D; o_qkv.scatter[1] = 1;
+  o_qkv.ptr[2] = vdst;    o_qkv.ld[2] = D; o_qkv.scatter[2] = 1;
+  o_qkv.seg_cols = D; o_qkv.idx = d_idx; o_qkv.n_sel = n_sel; o_qkv.n_rows = N;
+  HERO_TRY(run_gemm(c, c->ws_a, w.w_qkv, w.b_qkv, M, 3 * D, D, o_qkv));
+  HERO_TRY(run_attention(c, c->ws_q, kdst, vdst, c->ws_o, n_sel));
+  GemmOut o_attn = {};
+  o_attn.ptr[0] = ga; o_attn.ld[0] = D; o_attn.scatter[0] = 1;
+  o_attn.seg_cols = D; o_attn.idx = d_idx; o_attn.n_sel = n_sel; o_attn.n_rows = N;
+  o_attn.gate = gate1; o_attn.gate_ld = mod_ld;
+  HERO_TRY(run_gemm(c, c->ws_o, w.w_o, w.b_o, M, D, D, o_attn));
+
+  // FFN branch: its input rows are x + G_attn (the residual add is applied to x once, below)
+  HERO_TRY(launch_gather_ln_modulate(d_x, ga, d_idx, shift2, scale2, mod_ld, c->ws_a, B, N, n_sel, D, 1e-5f,
+                                     g.dtype, c->stream));
+  GemmOut o_up = {};
+  o_up.ptr[0] = c->ws_u; o_up.ld[0] = F; o_up.scatter[0] = 0;
+  o_up.seg_cols = F; o_up.idx = d_idx; o_up.n_sel = n_sel; o_up.n_rows = N; o_up.act = 1;
+  HERO_TRY(run_gemm(c, c->ws_a, w.w_1, w.b_1, M, F, D, o_up));
+  GemmOut o_dn = {};
+  o_dn.ptr[0] = gf; o_dn.ld[0] = D; o_dn.scatter[0] = 1;
+  o_dn.seg_cols = D; o_dn.idx = d_idx; o_dn.n_sel = n_sel; o_dn.n_rows = N;
+  o_dn.gate = gate2; o_dn.gate_ld = mod_ld;
+  HERO_TRY(run_gemm(c, c->ws_u, w.w_2, w.b_2, M, D, F, o_dn));
+
+  // x = (x + G_attn) + G_ffn for every row: fresh rows and cached rows alike
+  HERO_TRY(launch_residual2(d_x, ga, gf, c->elems, g.dtype, c->stream));
+
+  if (full) {
+    if (deep) {
+      bm.last_slot = new_slot;
+      if (bm.n_hist < 2) bm.n_hist++;
+    } else {
+      HERO_CUDA_TRY(cudaMemsetAsync(bm.ages[bm.ages_cur], 0, (size_t)c->n_video * sizeof(uint16_t), c->stream));
+    }
+  }
+  return HERO_OK;
+}
+
+int extrapolate_block(hero_ctx* c, int block, void* d_x, int k, int d) {
+  BlockMem& bm = c->blk[block];
+  if (bm.n_hist == 0) return HERO_ERR_STATE;
+  const int last = bm.last_slot, prev = bm.n_hist >= 2 ? (last ^ 1) : last;   // one slot only: Delta = 0
+  return launch_extrapolate_residual(d_x, bm.hist[0][prev], bm.hist[0][last], bm.hist[1][prev], bm.hist[1][last],
+                                     c->elems, k, d, c->cfg.dtype, c->stream);
+}
+
+int validate(const hero_config* g) {
+  if (g->n_blocks <= 0 || g->n_shallow < 0 || g->n_shallow > g->n_blocks) return HERO_ERR_ARG;
+  if (g->hidden <= 0 || g->n_heads <= 0 || g->head_dim <= 0 || g->hidden != g->n_heads * g->head_dim) return HERO_ERR_ARG;
+  if (g->ffn_dim <= 0 || g->temb_dim <= 0) return HERO_ERR_ARG;
+  if (g->batch <= 0 || g->batch > 8 || g->frames <= 0 || g->grid_h <= 0 || g->grid_w <= 0 || g->n_text < 0) return HERO_ERR_ARG;
+  if (g->patch_h <= 0 || g->patch_w <= 0) return HERO_ERR_ARG;
+  if (g->ratio_num <= 0 || g->ratio_den <= 0 || g->ratio_num > g->ratio_den) return HERO_ERR_ARG;
+  if (g->quota_mode != 0 && g->quota_mode != 1) return HERO_ERR_ARG;
+  if (g->warmup_full_steps < 1 || g->full_interval < 0) return HERO_ERR_ARG;
+  if (g->dtype != HERO_DTYPE_FP32 && g->dtype != HERO_DTYPE_BF16) return HERO_ERR_ARG;
+  if (g->n_shallow > kMaxSelectBatch) return HERO_ERR_ARG;
+  if (g->dtype == HERO_DTYPE_BF16) {
+    if (g->head_dim != 64 || g->hidden % 8 || g->ffn_dim % 8 || g->temb_dim % 8) return HERO_ERR_ALIGN;
+  } else {
+    if (g->head_dim != 32 && g->head_dim != 64 && g->head_dim != 128) return HERO_ERR_ARG;
+    if (g->hidden % 4 || g->ffn_dim % 4 || g->temb_dim % 4) return HERO_ERR_ALIGN;
+  }
+  const long long n_video = (long long)g->frames * g->grid_h * g->grid_w;
+  if (n_video + g->n_text > (1ll << 30)) return HERO_ERR_ARG;
+  return HERO_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* hero_strerror(int code) {
+  switch (code) {
+    case HERO_OK: return "ok";
+    case HERO_ERR_ARG: return "invalid argument";
+    case HERO_ERR_ALIGN: return "pointer or dimension not 16-byte aligned";
+    case HERO_ERR_CAP: return "index list capacity too small";
+    case HERO_ERR_STATE: return "call order violated";
+    case HERO_ERR_CUDA: return "CUDA call failed";
+    case HERO_ERR_TIMEOUT: return "bounded device wait ran out";
+    case HERO_ERR_NOMEM: return "device allocation failed";
+    default: return "unknown error";
+  }
+}
+
+const char* hero_last_cuda_error(void) { return g_last_error.c_str(); }
+
+void hero_destroy(hero_ctx* c) {
+  if (!c) return;
+  if (c->stream) cudaStreamSynchronize(c->stream); else cudaDeviceSynchronize();
+  for (void* p : c->allocs) cudaFree(p);
+  delete c;
+}
+
+int hero_init(hero_ctx** out, const hero_config* cfg, const hero_block_weights* blocks, void* cuda_stream) {
+  if (!out || !cfg || !blocks) return HERO_ERR_ARG;
+  *out = nullptr;
+  HERO_TRY(validate(cfg));
+  for (int l = 0; l < cfg->n_blocks; ++l) {
+    const void* ps[10] = {blocks[l].w_mod, blocks[l].b_mod, blocks[l].w_qkv, blocks[l].b_qkv, blocks[l].w_o,
+                          blocks[l].b_o,   blocks[l].w_1,   blocks[l].b_1,   blocks[l].w_2,   blocks[l].b_2};
+    for (const void* p : ps) {
+      if (!p) return HERO_ERR_ARG;
+      if (!aligned16(p)) return HERO_ERR_ALIGN;
+    }
+  }
+  if (cfg->dtype == HERO_DTYPE_BF16) HERO_TRY(tc_init_driver_api());
+  hero_ctx* c = new (std::nothrow) hero_ctx();
+  if (!c) return HERO_ERR_NOMEM;
+  c->cfg = *cfg;
+  c->stream = (cudaStream_t)cuda_stream;
+  c->n_video = cfg->frames * cfg->grid_h * cfg->grid_w;
+  c->N = cfg->n_text + c->n_video;
+  c->n_mod = cfg->has_gate ? 6 : 4;
+  c->esz = dtype_size(cfg->dtype);
+  c->elems = (long long)cfg->batch * c->N * cfg->hidden;
+  c->idx_cap = c->n_video;
+  c->mode1_n_sel = mode1_total(*cfg);
+  c->w.assign(blocks, blocks + cfg->n_blocks);
+  c->blk.resize(cfg->n_blocks);
+  const size_t tensor = (size_t)c->elems * c->esz;
+  int rc = HERO_OK;
+  auto A = [&](void** p, size_t bytes) { if (rc == HERO_OK) rc = dev_alloc(c, p, bytes); };
+  for (int l = 0; l < cfg->n_blocks && rc == HERO_OK; ++l) {
+    BlockMem& bm = c->blk[l];
+    if (l < cfg->n_shallow) {
+      A(&bm.k, tensor); A(&bm.v, tensor); A(&bm.g[0], tensor); A(&bm.g[1], tensor);
+      A((void**)&bm.ages[0], (size_t)c->n_video * 2); A((void**)&bm.ages[1], (size_t)c->n_video * 2);
+    } else {
+      for (int br = 0; br < 2; ++br) for (int s = 0; s < 2; ++s) A(&bm.hist[br][s], tensor);
+    }
+  }
+  if (cfg->n_shallow < cfg->n_blocks) { A(&c->kv_tmp[0], tensor); A(&c->kv_tmp[1], tensor); }
+  A(&c->ws_a, tensor); A(&c->ws_q, tensor); A(&c->ws_o, tensor);
+  A(&c->ws_u, (size_t)cfg->batch * c->N * cfg->ffn_dim * c->esz);
+  A((void**)&c->mod, (size_t)cfg->batch * c->n_mod * cfg->hidden * sizeof(float));
+  A((void**)&c->idx_ws, (size_t)(cfg->n_shallow > 0 ? cfg->n_shallow : 1) * c->idx_cap * sizeof(int));
+  A((void**)&c->d_status, 16);
+  A(&c->x_stage, tensor);
+  A(&c->temb_stage, (size_t)cfg->batch * cfg->temb_dim * c->esz);
+  if (rc != HERO_OK) { hero_destroy(c); return rc; }
+  cudaError_t e = cudaMemsetAsync(c->d_status, 0, 16, c->stream);
+  if (e != cudaSuccess) { set_cuda_error(e, "cudaMemsetAsync"); hero_destroy(c); return HERO_ERR_CUDA; }
+  rc = hero_reset(c);
+  if (rc != HERO_OK) { hero_destroy(c); return rc; }
+  *out = c;
+  return HERO_OK;
+}
+
+int hero_reset(hero_ctx* c) {
+  if (!c) return HERO_ERR_ARG;
+  for (int l = 0; l < c->cfg.n_blocks; ++l) {
+    BlockMem& bm = c->blk[l];
+    bm.calls = 0; bm.ages_cur = 0; bm.n_hist = 0; bm.last_slot = 0;
+    if (bm.ages[0]) HERO_CUDA_TRY(cudaMemsetAsync(bm.ages[0], 0, (size_t)c->n_video * 2, c->stream));
+    if (bm.ages[1]) HERO_CUDA_TRY(cudaMemsetAsync(bm.ages[1], 0, (size_t)c->n_video * 2, c->stream));
+  }
+  c->n_full = 0; c->s_prev = 0; c->s_last = 0;
+  return HERO_OK;
+}
+
+long long hero_device_bytes(const hero_ctx* c) { return c ? c->bytes : 0; }
+
+int hero_check_status(hero_ctx* c) {
+  if (!c) return HERO_ERR_ARG;
+  int st[4] = {0, 0, 0, 0};
+  HERO_CUDA_TRY(cudaMemcpyAsync(st, c->d_status, 16, cudaMemcpyDeviceToHost, c->stream));
+  HERO_CUDA_TRY(cudaStreamSynchronize(c->stream));
+  if (st[0] != 0) {
+    cudaMemsetAsync(c->d_status, 0, 16, c->stream);
+    return HERO_ERR_TIMEOUT;
+  }
+  return HERO_OK;
+}
+
+int hero_next_n_sel(const hero_ctx* c, int block) {
+  if (!c || block < 0 || block >= c->cfg.n_shallow) return HERO_ERR_ARG;
+  return n_sel_for_call(c, c->blk[block].calls);
+}
+
+int hero_select_tokens(hero_ctx* c, int block, int* d_idx, int cap, int* n_sel) {
+  if (!c || !d_idx) return HERO_ERR_ARG;
+  if (block < 0 || block >= c->cfg.n_shallow) return HERO_ERR_ARG;
+  BlockMem& bm = c->blk[block];
+  const int n = n_sel_for_call(c, bm.calls);
+  if (cap < n) return HERO_ERR_CAP;
+  SelectBatch batch;
+  batch.n = 1;
+  batch.block[0] = block; batch.call[0] = bm.calls;
+  batch.ages_in[0] = bm.ages[bm.ages_cur]; batch.ages_out[0] = bm.ages[bm.ages_cur ^ 1];
+  batch.idx[0] = d_idx;
+  HERO_TRY(launch_select(geom_of(c->cfg), batch, c->stream));
+  bm.ages_cur ^= 1;
+  bm.calls++;
+  if (n_sel) *n_sel = n;
+  return HERO_OK;
+}
+
+int hero_refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, const int* d_idx, int n_sel) {
+  if (!c || !d_x || !d_temb) return HERO_ERR_ARG;
+  if (block < 0 || block >= c->cfg.n_blocks) return HERO_ERR_ARG;
+  if (!aligned16(d_x) || !aligned16(d_temb)) return HERO_ERR_ALIGN;
+  if (d_idx == nullptr) {
+    if (n_sel != c->N) return HERO_ERR_ARG;
+  } else {
+    if (n_sel < 0 || n_sel > c->N) return HERO_ERR_ARG;
+    if (block >= c->cfg.n_shallow) return HERO_ERR_ARG;   // deep blocks keep no K/V cache to refresh against
+    if (n_sel == 0) {                                      // nothing refreshed: the residual adds still happen
+      BlockMem& bm = c->blk[block];
+      return launch_residual2(d_x, bm.g[0], bm.g[1], c->elems, c->cfg.dtype, c->stream);
+    }
+  }
+  return refresh_block(c, block, d_x, d_temb, d_idx, n_sel);
+}
+
+int hero_extrapolate_block(hero_ctx* c, int block, void* d_x, int k, int d) {
+  if (!c || !d_x) return HERO_ERR_ARG;
+  if (block < c->cfg.n_shallow || block >= c->cfg.n_blocks) return HERO_ERR_ARG;
+  if (k < 0 || d <= 0) return HERO_ERR_ARG;
+  if (!aligned16(d_x)) return HERO_ERR_ALIGN;
+  return extrapolate_block(c, block, d_x, k, d);
+}
+
+int hero_is_full_step(const hero_ctx* c, int step) {
+  if (!c || step < 0) return HERO_ERR_ARG;
+  return is_full(c->cfg, step) ? 1 : 0;
+}
+
+int hero_step(hero_ctx* c, int step, void* d_x, const void* d_temb) {
+  if (!c || !d_x || !d_temb || step < 0) return HERO_ERR_ARG;
+  if (!aligned16(d_x) || !aligned16(d_temb)) return HERO_ERR_ALIGN;
+  const hero_config& g = c->cfg;
+  if (is_full(g, step)) {
+    for (int l = 0; l < g.n_blocks; ++l) HERO_TRY(refresh_block(c, l, d_x, d_temb, nullptr, c->N));
+    c->s_prev = c->s_last; c->s_last = step; c->n_full++;
+    return HERO_OK;
+  }
+  if (c->n_full == 0) return HERO_ERR_STATE;
+  const int k = step - c->s_last;
+  const int d = c->n_full >= 2 ? c->s_last - c->s_prev : 1;
+  if (k <= 0 || d <= 0) return HERO_ERR_STATE;
+  // all shallow blocks draw their lists in one launch: the draw depends on counters only
+  int n_sel[kMaxSelectBatch];
+  if (g.n_shallow > 0) {
+    SelectBatch batch;
+    batch.n = g.n_shallow;
+    for (int l = 0; l < g.n_shallow; ++l) {
+      BlockMem& bm = c->blk[l];
+      n_sel[l] = n_sel_for_call(c, bm.calls);
+      batch.block[l] = l; batch.call[l] = bm.calls;
+      batch.ages_in[l] = bm.ages[bm.ages_cur]; batch.ages_out[l] = bm.ages[bm.ages_cur ^ 1];
+      batch.idx[l] = c->idx_ws + (size_t)l * c->idx_cap;
+    }
+    HERO_TRY(launch_select(geom_of(g), batch, c->stream));
+    for (int l = 0; l < g.n_shallow; ++l) { c->blk[l].ages_cur ^= 1; c->blk[l].calls++; }
+  }
+  for (int l = 0; l < g.n_blocks; ++l) {
+    if (l < g.n_shallow) {
+      if (n_sel[l] > 0) {
+        HERO_TRY(refresh_block(c, l, d_x, d_temb, c->idx_ws + (size_t)l * c->idx_cap, n_sel[l]));
+      } else {
+        HERO_TRY(launch_residual2(d_x, c->blk[l].g[0], c->blk[l].g[1], c->elems, g.dtype, c->stream));
+      }
+    } else {
+      HERO_TRY(extrapolate_block(c, l, d_x, k, d));
+    }
+  }
+  return HERO_OK;
+}
+
+int hero_step_host(hero_ctx* c, int step, void* h_x, const void* h_temb) {
+  if (!c || !h_x || !h_temb) return HERO_ERR_ARG;
+  const size_t xb = (size_t)c->elems * c->esz, tb = (size_t)c->cfg.batch * c->cfg.temb_dim * c->esz;
+  HERO_CUDA_TRY(cudaMemcpyAsync(c->x_stage, h_x, xb, cudaMemcpyHostToDevice, c->stream));
+  HERO_CUDA_TRY(cudaMemcpyAsync(c->temb_stage, h_temb, tb, cudaMemcpyHostToDevice, c->stream));
+  HERO_TRY(hero_step(c, step, c->x_stage, c->temb_stage));
+  HERO_CUDA_TRY(cudaMemcpyAsync(h_x, c->x_stage, xb, cudaMemcpyDeviceToHost, c->stream));
+  HERO_CUDA_TRY(cudaStreamSynchronize(c->stream));
+  return HERO_OK;
+}
+
+// ---------------------------------------------------------------- isolated kernels
+int hero_extrapolate(const void* g_prev, const void* g_last, void* out, long long n, int k, int d, int dtype,
+                     void* stream) {
+  if (n < 0 || d <= 0 || k < 0) return HERO_ERR_ARG;
+  if (dtype != HERO_DTYPE_FP32 && dtype != HERO_DTYPE_BF16) return HERO_ERR_ARG;
+  if (n == 0) return HERO_OK;
+  if (!g_prev || !g_last || !out) return HERO_ERR_ARG;
+  if (!aligned16(g_prev) || !aligned16(g_last) || !aligned16(out)) return HERO_ERR_ALIGN;
+  return launch_extrapolate(g_prev, g_last, out, n, k, d, dtype, (cudaStream_t)stream);
+}
+
+static int check_rows(const void* src, const int* idx, void* dst, int B, int N, int n_sel, int D, int dtype) {
+  if (B < 0 || N < 0 || n_sel < 0 || D <= 0 || n_sel > N) return HERO_ERR_ARG;
+  if (dtype != HERO_DTYPE_FP32 && dtype != HERO_DTYPE_BF16) return HERO_ERR_ARG;
+  if (B == 0 || n_sel == 0) return HERO_OK;
+  if (!src || !idx || !dst) return HERO_ERR_ARG;
+  if (!aligned16(src) || !aligned16(dst)) return HERO_ERR_ALIGN;
+  return 1;
+}
+int hero_gather_rows(const void* src, const int* idx, void* dst, int B, int N, int n_sel, int D, int dtype,
+                     void* stream) {
+  const int r = check_rows(src, idx, dst, B, N, n_sel, D, dtype);
+  if (r <= 0) return r;
+  return launch_gather_rows(src, idx, dst, B, N, n_sel, D, dtype, (cudaStream_t)stream);
+}
+int hero_scatter_rows(const void* src, const int* idx, void* dst, int B, int N, int n_sel, int D, int dtype,
+                      void* stream) {
+  const int r = check_rows(src, idx, dst, B, N, n_sel, D, dtype);
+  if (r <= 0) return r;
+  return launch_scatter_rows(src, idx, dst, B, N, n_sel, D, dtype, (cudaStream_t)stream);
+}
+
+// The isolated tensor-core calls own a status word each; a timeout is reported on the next call.
+static int* isolated_status() {
+  static int* p = nullptr;
+  if (!p) {
+    if (cudaMalloc((void**)&p, 16) != cudaSuccess) { p = nullptr; return nullptr; }
+    cudaMemset(p, 0, 16);
+  }
+  return p;
+}
+static int poll_isolated_status(cudaStream_t s) {
+  int* p = isolated_status();
+  if (!p) return HERO_ERR_NOMEM;
+  int st = 0;
+  HERO_CUDA_TRY(cudaMemcpyAsync(&st, p, 4, cudaMemcpyDeviceToHost, s));
+  HERO_CUDA_TRY(cudaStreamSynchronize(s));
+  if (st) { cudaMemset(p, 0, 16); return HERO_ERR_TIMEOUT; }
+  return HERO_OK;
+}
+
+int hero_gemm_bf16(const void* a, const void* w, const void* bias, void* cmat, int M, int N, int K, int act,
+                   void* stream) {
+  if (M < 0 || N <= 0 || K <= 0 || (act != 0 && act != 1)) return HERO_ERR_ARG;
+  if (M == 0) return HERO_OK;
+  if (!a || !w || !bias || !cmat) return HERO_ERR_ARG;
+  int* st = isolated_status();
+  if (!st) return HERO_ERR_NOMEM;
+  GemmOut o = {};
+  o.ptr[0] = cmat; o.ld[0] = N; o.scatter[0] = 0;
+  o.seg_cols = (N + 31) / 32 * 32; o.n_sel = M; o.n_rows = M; o.act = act;
+  return launch_tc_gemm(a, w, bias, M, N, K, o, st, (cudaStream_t)stream);
+}
+
+int hero_attention_bf16(const void* q, const void* k, const void* v, void* o, int B, int n_q, int N, int heads,
+                        void* stream) {
+  if (B < 0 || n_q < 0 || N <= 0 || heads <= 0) return HERO_ERR_ARG;
+  if (B == 0 || n_q == 0) return HERO_OK;
+  if (!q || !k || !v || !o) return HERO_ERR_ARG;
+  int* st = isolated_status();
+  if (!st) return HERO_ERR_NOMEM;
+  return launch_tc_attention(q, k, v, o, B, n_q, N, heads, st, (cudaStream_t)stream);
+}
+
+// Synchronise `stream` and report whether an isolated tensor-core call gave up on a wait.
+int hero_isolated_status(void* stream) { return poll_isolated_status((cudaStream_t)stream); }
+
+// ---------------------------------------------------------------- state access
+static int state_ptr(hero_ctx* c, int block, int what, void** p, size_t* bytes) {
+  const hero_config& g = c->cfg;
+  if (what == HERO_STATE_STEPS) { *p = nullptr; *bytes = 12; return HERO_OK; }
+  if (block < 0 || block >= g.n_blocks) return HERO_ERR_ARG;
+  BlockMem& bm = c->blk[block];
+  const bool deep = block >= g.n_shallow;
+  const size_t tensor = (size_t)c->elems * c->esz;
+  switch (what) {
+    case HERO_STATE_AGES: if (deep) return HERO_ERR_ARG; *p = bm.ages[bm.ages_cur]; *bytes = (size_t)c->n_video * 2; return HERO_OK;
+    case HERO_STATE_CALLS: *p = nullptr; *bytes = 4; return HERO_OK;
+    case HERO_STATE_K: if (deep) return HERO_ERR_ARG; *p = bm.k; *bytes = tensor; return HERO_OK;
+    case HERO_STATE_V: if (deep) return HERO_ERR_ARG; *p = bm.v; *bytes = tensor; return HERO_OK;
+    case HERO_STATE_G_ATTN: *p = deep ? bm.hist[0][bm.last_slot] : bm.g[0]; *bytes = tensor; return HERO_OK;
+    case HERO_STATE_G_FFN: *p = deep ? bm.hist[1][bm.last_slot] : bm.g[1]; *bytes = tensor; return HERO_OK;
+    case HERO_STATE_G_ATTN_PREV: if (!deep) return HERO_ERR_ARG; *p = bm.hist[0][bm.last_slot ^ 1]; *bytes = tensor; return HERO_OK;
+    case HERO_STATE_G_FFN_PREV: if (!deep) return HERO_ERR_ARG; *p = bm.hist[1][bm.last_slot ^ 1]; *bytes = tensor; return HERO_OK;
+    default: return HERO_ERR_ARG;
+  }
+}
+
+int hero_state_get(hero_ctx* c, int block, int what, void* h_out, long long bytes) {
+  if (!c || !h_out) return HERO_ERR_ARG;
+  void* p; size_t need;
+  HERO_TRY(state_ptr(c, block, what, &p, &need));
+  if (bytes != (long long)need) return HERO_ERR_ARG;
+  if (what == HERO_STATE_STEPS) { int v[3] = {c->n_full, c->s_prev, c->s_last}; memcpy(h_out, v, 12); return HERO_OK; }
+  if (what == HERO_STATE_CALLS) { memcpy(h_out, &c->blk[block].calls, 4); return HERO_OK; }
+  HERO_CUDA_TRY(cudaMemcpyAsync(h_out, p, need, cudaMemcpyDeviceToHost, c->stream));
+  HERO_CUDA_TRY(cudaStreamSynchronize(c->stream));
+  return HERO_OK;
+}
+
+int hero_state_set(hero_ctx* c, int block, int what, const void* h_in, long long bytes) {
+  if (!c || !h_in) return HERO_ERR_ARG;
+  void* p; size_t need;
+  HERO_TRY(state_ptr(c, block, what, &p, &need));
+  if (bytes != (long long)need) return HERO_ERR_ARG;
+  if (what == HERO_STATE_STEPS) {
+    int v[3]; memcpy(v, h_in, 12);
+    if (v[0] < 0) return HERO_ERR_ARG;
+    c->n_full = v[0]; c->s_prev = v[1]; c->s_last = v[2];
+    return HERO_OK;
+  }
+  if (what == HERO_STATE_CALLS) { int v; memcpy(&v, h_in, 4); if (v < 0) return HERO_ERR_ARG; c->blk[block].calls = v; return HERO_OK; }
+  HERO_CUDA_TRY(cudaMemcpyAsync(p, h_in, need, cudaMemcpyHostToDevice, c->stream));
+  HERO_CUDA_TRY(cudaStreamSynchronize(c->stream));
+  if (block >= c->cfg.n_shallow) {   // planting a deep block's history marks the slots as valid
+    BlockMem& bm = c->blk[block];
+    if (what == HERO_STATE_G_ATTN || what == HERO_STATE_G_FFN) { if (bm.n_hist < 1) bm.n_hist = 1; }
+    if (what == HERO_STATE_G_ATTN_PREV || what == HERO_STATE_G_FFN_PREV) bm.n_hist = 2;
+  }
+  return HERO_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,110 @@
+// Internal declarations shared by the translation units of libhero.so.
+// Nothing here is part of the public ABI (see include/hero.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "hero.h"
+
+namespace hero {
+
+// ---------------------------------------------------------------------------
+// Error plumbing
+// ---------------------------------------------------------------------------
+void set_cuda_error(cudaError_t e, const char* what);
+#define HERO_CUDA_TRY(expr)                                  \
+  do {                                                       \
+    cudaError_t e__ = (expr);                                \
+    if (e__ != cudaSuccess) {                                \
+      ::hero::set_cuda_error(e__, #expr);                    \
+      return HERO_ERR_CUDA;                                  \
+    }                                                        \
+  } while (0)
+#define HERO_TRY(expr)                  \
+  do {                                  \
+    int r__ = (expr);                   \
+    if (r__ != HERO_OK) return r__;     \
+  } while (0)
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static inline size_t dtype_size(int dtype) { return dtype == HERO_DTYPE_BF16 ? 2 : 4; }
+
+// ---------------------------------------------------------------------------
+// Where a GEMM's output goes (Eq. 3's merge happens in the epilogue).
+// The N dimension is cut into up to three segments of seg_cols columns (q | k | v for the
+// QKV projection, one segment otherwise).  Row m of the compact operand belongs to batch
+// b = m / n_sel and list position i = m % n_sel; a scattered segment writes it to row
+// b * n_rows + (idx ? idx[i] : i) of its destination, a compact segment to row m.
+// ---------------------------------------------------------------------------
+struct GemmOut {
+  void* ptr[3];
+  long long ld[3];
+  int scatter[3];
+  int seg_cols;
+  const int* idx;
+  int n_sel;
+  int n_rows;
+  const float* gate;   // optional multiplier [B, gate_ld], indexed by column within the segment
+  int gate_ld;
+  int act;             // 0 = identity, 1 = GELU-tanh
+};
+
+// Geometry of the selection problem (Sec. 4.3).
+struct SelectGeom {
+  int frames, grid_h, grid_w, n_text;
+  int patch_h, patch_w;
+  int ratio_num, ratio_den, quota_mode;
+  uint32_t seed_lo;
+};
+constexpr int kMaxSelectBatch = 64;
+struct SelectBatch {
+  int n;                                  // number of blocks selected in this launch
+  int block[kMaxSelectBatch];             // block id (enters the hash)
+  int call[kMaxSelectBatch];              // per-block call counter value
+  const uint16_t* ages_in[kMaxSelectBatch];
+  uint16_t* ages_out[kMaxSelectBatch];
+  int* idx[kMaxSelectBatch];
+};
+
+// ---------------------------------------------------------------------------
+// Kernel launchers (each returns HERO_OK or HERO_ERR_CUDA; all asynchronous)
+// ---------------------------------------------------------------------------
+int launch_select(const SelectGeom& g, const SelectBatch& batch, cudaStream_t s);
+
+int launch_extrapolate(const void* g_prev, const void* g_last, void* out, long long n, int k, int d,
+                       int dtype, cudaStream_t s);
+// x += e(attn history) ; x += e(ffn history)
+int launch_extrapolate_residual(void* x, const void* ga_prev, const void* ga_last, const void* gf_prev,
+                                const void* gf_last, long long n, int k, int d, int dtype, cudaStream_t s);
+// x = (x + ga) + gf
+int launch_residual2(void* x, const void* ga, const void* gf, long long n, int dtype, cudaStream_t s);
+int launch_gather_rows(const void* src, const int* idx, void* dst, int B, int N, int n_sel, int D,
+                       int dtype, cudaStream_t s);
+int launch_scatter_rows(const void* src, const int* idx, void* dst, int B, int N, int n_sel, int D,
+                        int dtype, cudaStream_t s);
+// mod[b, j] = b_mod[j] + sum_e silu(temb[b,e]) * w_mod[j,e]   (fp32 output)
+int launch_modulation(const void* temb, const void* w_mod, const void* b_mod, float* mod, int B,
+                      int n_out, int E, int dtype, cudaStream_t s);
+// a[m,:] = LN(x[row(m),:] (+ add[row(m),:])) * (1 + scale[b,:]) + shift[b,:]
+int launch_gather_ln_modulate(const void* x, const void* add, const int* idx, const float* shift,
+                              const float* scale, int mod_ld, void* a, int B, int N, int n_sel, int D,
+                              float eps, int dtype, cudaStream_t s);
+
+// fp32 / generic CUDA-core path (config 1 runs in fp32, where tensor cores would break parity)
+int launch_simt_gemm(const void* a, const void* w, const void* bias, int M, int Nout, int K,
+                     const GemmOut& out, int dtype, cudaStream_t s);
+int launch_simt_attention(const void* q, const void* k, const void* v, void* o, int B, int n_q, int N,
+                          int heads, int head_dim, int dtype, cudaStream_t s);
+
+// bf16 tensor-core path (tcgen05 + TMEM + TMA)
+int tc_init_driver_api();   // resolves cuTensorMapEncodeTiled once
+int launch_tc_gemm(const void* a, const void* w, const void* bias, int M, int Nout, int K,
+                   const GemmOut& out, int* d_status, cudaStream_t s);
+int launch_tc_attention(const void* q, const void* k, const void* v, void* o, int B, int n_q, int N,
+                        int heads, int* d_status, cudaStream_t s);
+
+int num_sms();
+
+}  // namespace hero

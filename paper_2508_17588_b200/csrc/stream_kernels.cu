@@ -1,0 +1,456 @@
+// HBM-bound kernels of the cached step: linear extrapolation (Eq. 5), residual adds
+// (Algorithm 1), row gather / scatter (Eq. 3's merge), the adaLN modulation vectors and the
+// fused gather + LayerNorm + modulate prologue of Eq. 2.  All of them move each byte once
+// with 128-bit accesses; grids are sized in multiples of the SM count.
+#include "hero_internal.h"
+
+namespace hero {
+
+int num_sms() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  }
+  return n;
+}
+
+namespace {
+
+// ------------------------------------------------------------------ 128-bit packets
+template <typename T>
+struct Vec;  // 16 bytes of T
+template <>
+struct Vec<float> {
+  static constexpr int N = 4;
+  float4 raw;
+  __device__ __forceinline__ void unpack(float (&f)[4]) const {
+    f[0] = raw.x; f[1] = raw.y; f[2] = raw.z; f[3] = raw.w;
+  }
+  __device__ __forceinline__ void pack(const float (&f)[4]) { raw = make_float4(f[0], f[1], f[2], f[3]); }
+};
+template <>
+struct Vec<__nv_bfloat16> {
+  static constexpr int N = 8;
+  uint4 raw;
+  __device__ __forceinline__ void unpack(float (&f)[8]) const {
+    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      f[2 * i] = __uint_as_float(w[i] << 16);
+      f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+  }
+  __device__ __forceinline__ void pack(const float (&f)[8]) {
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const __nv_bfloat162 p = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+      w[i] = *reinterpret_cast<const uint32_t*>(&p);
+    }
+    raw = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+};
+
+template <typename T>
+__device__ __forceinline__ float to_f(T v);
+template <>
+__device__ __forceinline__ float to_f<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T>
+__device__ __forceinline__ T from_f(float v);
+template <>
+__device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// streaming loads/stores: these tensors are touched once per step, keep them out of L1
+template <typename V>
+__device__ __forceinline__ V ld_stream(const V* p) {
+  V v;
+  v.raw = __ldcs(&p->raw);
+  return v;
+}
+template <typename V>
+__device__ __forceinline__ void st_stream(V* p, const V& v) { __stcs(&p->raw, v.raw); }
+
+constexpr int kStreamThreads = 256;
+constexpr int kStreamUnroll = 2;
+
+static inline int stream_grid(long long n_vec) {
+  const long long per_block = (long long)kStreamThreads * kStreamUnroll;
+  long long blocks = (n_vec + per_block - 1) / per_block;
+  const long long cap = (long long)num_sms() * 16;   // grid-stride beyond 16 CTAs per SM
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  return (int)blocks;
+}
+
+// ------------------------------------------------------------------ Eq. 5
+// e = g_last + (g_last - g_prev) * (k/d), evaluated as one fp32 FMA per element.
+template <typename T>
+__global__ void __launch_bounds__(kStreamThreads) extrapolate_kernel(const T* __restrict__ g_prev,
+                                                                     const T* __restrict__ g_last,
+                                                                     T* __restrict__ out, long long n, float c) {
+  using V = Vec<T>;
+  const long long n_vec = n / V::N;
+  const V* p = reinterpret_cast<const V*>(g_prev);
+  const V* l = reinterpret_cast<const V*>(g_last);
+  V* o = reinterpret_cast<V*>(out);
+  const long long stride = (long long)gridDim.x * kStreamThreads * kStreamUnroll;
+  for (long long i0 = (long long)blockIdx.x * kStreamThreads * kStreamUnroll + threadIdx.x; i0 < n_vec; i0 += stride) {
+    V vp[kStreamUnroll], vl[kStreamUnroll];
+#pragma unroll
+    for (int u = 0; u < kStreamUnroll; ++u) {
+      const long long i = i0 + (long long)u * kStreamThreads;
+      if (i < n_vec) { vp[u] = ld_stream(p + i); vl[u] = ld_stream(l + i); }
+    }
+#pragma unroll
+    for (int u = 0; u < kStreamUnroll; ++u) {
+      const long long i = i0 + (long long)u * kStreamThreads;
+      if (i < n_vec) {
+        float fp[V::N], fl[V::N];
+        vp[u].unpack(fp); vl[u].unpack(fl);
+#pragma unroll
+        for (int j = 0; j < V::N; ++j) fl[j] = fmaf(fl[j] - fp[j], c, fl[j]);
+        V r; r.pack(fl);
+        st_stream(o + i, r);
+      }
+    }
+  }
+  // ragged tail (fewer than one packet)
+  const long long tail0 = n_vec * V::N;
+  if (blockIdx.x == 0 && threadIdx.x < n - tail0) {
+    const long long i = tail0 + threadIdx.x;
+    const float a = to_f(g_last[i]), b = to_f(g_prev[i]);
+    out[i] = from_f<T>(fmaf(a - b, c, a));
+  }
+}
+
+// x += e(attn) ; x += e(ffn)  (both branches of a deep block in one pass: 5 reads, 1 write)
+template <typename T>
+__global__ void __launch_bounds__(kStreamThreads)
+extrapolate_residual_kernel(T* __restrict__ x, const T* __restrict__ ga_prev, const T* __restrict__ ga_last,
+                            const T* __restrict__ gf_prev, const T* __restrict__ gf_last, long long n, float c) {
+  using V = Vec<T>;
+  const long long n_vec = n / V::N;
+  V* xv = reinterpret_cast<V*>(x);
+  const V* ap = reinterpret_cast<const V*>(ga_prev);
+  const V* al = reinterpret_cast<const V*>(ga_last);
+  const V* fp_ = reinterpret_cast<const V*>(gf_prev);
+  const V* fl_ = reinterpret_cast<const V*>(gf_last);
+  const long long stride = (long long)gridDim.x * kStreamThreads;
+  for (long long i = (long long)blockIdx.x * kStreamThreads + threadIdx.x; i < n_vec; i += stride) {
+    const V vx = ld_stream(xv + i), v1 = ld_stream(ap + i), v2 = ld_stream(al + i), v3 = ld_stream(fp_ + i),
+            v4 = ld_stream(fl_ + i);
+    float fx[V::N], f1[V::N], f2[V::N], f3[V::N], f4[V::N];
+    vx.unpack(fx); v1.unpack(f1); v2.unpack(f2); v3.unpack(f3); v4.unpack(f4);
+#pragma unroll
+    for (int j = 0; j < V::N; ++j) {
+      const float ea = fmaf(f2[j] - f1[j], c, f2[j]);
+      const float ef = fmaf(f4[j] - f3[j], c, f4[j]);
+      fx[j] = (fx[j] + ea) + ef;
+    }
+    V r; r.pack(fx);
+    st_stream(xv + i, r);
+  }
+  const long long tail0 = n_vec * V::N;
+  if (blockIdx.x == 0 && threadIdx.x < n - tail0) {
+    const long long i = tail0 + threadIdx.x;
+    const float a1 = to_f(ga_prev[i]), a2 = to_f(ga_last[i]), b1 = to_f(gf_prev[i]), b2 = to_f(gf_last[i]);
+    x[i] = from_f<T>((to_f(x[i]) + fmaf(a2 - a1, c, a2)) + fmaf(b2 - b1, c, b2));
+  }
+}
+
+// x = (x + ga) + gf  (both residual adds of a refresh block in one pass)
+template <typename T>
+__global__ void __launch_bounds__(kStreamThreads) residual2_kernel(T* __restrict__ x, const T* __restrict__ ga,
+                                                                   const T* __restrict__ gf, long long n) {
+  using V = Vec<T>;
+  const long long n_vec = n / V::N;
+  V* xv = reinterpret_cast<V*>(x);
+  const V* a = reinterpret_cast<const V*>(ga);
+  const V* f = reinterpret_cast<const V*>(gf);
+  const long long stride = (long long)gridDim.x * kStreamThreads * kStreamUnroll;
+  for (long long i0 = (long long)blockIdx.x * kStreamThreads * kStreamUnroll + threadIdx.x; i0 < n_vec; i0 += stride) {
+    V vx[kStreamUnroll], va[kStreamUnroll], vf[kStreamUnroll];
+#pragma unroll
+    for (int u = 0; u < kStreamUnroll; ++u) {
+      const long long i = i0 + (long long)u * kStreamThreads;
+      if (i < n_vec) { vx[u] = ld_stream(xv + i); va[u] = ld_stream(a + i); vf[u] = ld_stream(f + i); }
+    }
+#pragma unroll
+    for (int u = 0; u < kStreamUnroll; ++u) {
+      const long long i = i0 + (long long)u * kStreamThreads;
+      if (i < n_vec) {
+        float fx[V::N], fa[V::N], ff[V::N];
+        vx[u].unpack(fx); va[u].unpack(fa); vf[u].unpack(ff);
+#pragma unroll
+        for (int j = 0; j < V::N; ++j) fx[j] = (fx[j] + fa[j]) + ff[j];
+        V r; r.pack(fx);
+        st_stream(xv + i, r);
+      }
+    }
+  }
+  const long long tail0 = n_vec * V::N;
+  if (blockIdx.x == 0 && threadIdx.x < n - tail0) {
+    const long long i = tail0 + threadIdx.x;
+    x[i] = from_f<T>((to_f(x[i]) + to_f(ga[i])) + to_f(gf[i]));
+  }
+}
+
+// ------------------------------------------------------------------ gather / scatter of rows
+// One warp moves one row in 16-byte packets; GATHER reads row idx[i] and writes row i,
+// SCATTER the reverse.  Rows not listed are never touched.
+template <bool GATHER>
+__global__ void __launch_bounds__(256) move_rows_kernel(const uint4* __restrict__ src, const int* __restrict__ idx,
+                                                        uint4* __restrict__ dst, int B, int N, int n_sel,
+                                                        int row_vec) {
+  const long long warp_global = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const long long n_warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  const long long total = (long long)B * n_sel;
+  for (long long m = warp_global; m < total; m += n_warps) {
+    const int b = (int)(m / n_sel), i = (int)(m - (long long)b * n_sel);
+    const long long far = ((long long)b * N + idx[i]) * row_vec, near = m * row_vec;
+    const uint4* s = src + (GATHER ? far : near);
+    uint4* d = dst + (GATHER ? near : far);
+    for (int c = lane; c < row_vec; c += 32) __stcs(d + c, __ldcs(s + c));
+  }
+}
+
+// ------------------------------------------------------------------ adaLN modulation vectors
+// mod[b, j] = b_mod[j] + sum_e silu(temb[b, e]) * w_mod[j, e]; one warp per output column j,
+// the weight row is read once with 16-byte loads and reused for every batch item.
+constexpr int kModMaxB = 8;
+template <typename T>
+__global__ void __launch_bounds__(256) modulation_kernel(const T* __restrict__ temb, const T* __restrict__ w_mod,
+                                                         const T* __restrict__ b_mod, float* __restrict__ mod,
+                                                         int B, int n_out, int E) {
+  extern __shared__ float s_act[];   // [B, E] silu(temb)
+  for (int i = threadIdx.x; i < B * E; i += blockDim.x) {
+    const float t = to_f(temb[i]);
+    s_act[i] = t / (1.0f + expf(-t));
+  }
+  __syncthreads();
+  const int lane = threadIdx.x & 31;
+  const int warps_per_block = blockDim.x >> 5;
+  using V = Vec<T>;
+  for (int j = blockIdx.x * warps_per_block + (threadIdx.x >> 5); j < n_out; j += gridDim.x * warps_per_block) {
+    float acc[kModMaxB];
+#pragma unroll
+    for (int b = 0; b < kModMaxB; ++b) acc[b] = 0.f;
+    const V* wrow = reinterpret_cast<const V*>(w_mod + (long long)j * E);
+    for (int c = lane; c < E / V::N; c += 32) {
+      float wf[V::N];
+      V wv; wv.raw = __ldg(&wrow[c].raw);
+      wv.unpack(wf);
+#pragma unroll
+      for (int b = 0; b < kModMaxB; ++b) {
+        if (b < B) {
+#pragma unroll
+          for (int q = 0; q < V::N; ++q) acc[b] = fmaf(s_act[b * E + c * V::N + q], wf[q], acc[b]);
+        }
+      }
+    }
+#pragma unroll
+    for (int b = 0; b < kModMaxB; ++b) {
+      if (b < B) {
+        float v = acc[b];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+        if (lane == 0) mod[(long long)b * n_out + j] = v + to_f(b_mod[j]);
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------ gather + LayerNorm + modulate (Eq. 2 prologue)
+// One CTA per refreshed row: the row (plus, for the FFN branch, the not-yet-added attention
+// output of the same row) is read once into shared memory as fp32, mean and biased variance
+// are reduced in two passes over that copy, and the modulated row is written compactly.
+constexpr int kLnThreads = 256;
+__device__ __forceinline__ float block_sum(float v, float* red) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  __syncthreads();
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  float t = (lane < kLnThreads / 32) ? red[lane] : 0.f;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, o);
+  return t;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kLnThreads)
+gather_ln_modulate_kernel(const T* __restrict__ x, const T* __restrict__ add, const int* __restrict__ idx,
+                          const float* __restrict__ shift, const float* __restrict__ scale, int mod_ld,
+                          T* __restrict__ a, int N, int n_sel, int D, float eps) {
+  extern __shared__ float s_row[];   // [D]
+  __shared__ float red[kLnThreads / 32];
+  using V = Vec<T>;
+  const int m = blockIdx.x;
+  const int b = m / n_sel, i = m - b * n_sel;
+  const long long row = (long long)b * N + (idx ? idx[i] : i);
+  const V* xr = reinterpret_cast<const V*>(x + row * D);
+  const V* ar = add ? reinterpret_cast<const V*>(add + row * D) : nullptr;
+  const int n_vec = D / V::N;
+  float sum = 0.f;
+  for (int c = threadIdx.x; c < n_vec; c += kLnThreads) {
+    float f[V::N];
+    V v; v.raw = __ldg(&xr[c].raw);
+    v.unpack(f);
+    if (ar) {
+      float g[V::N];
+      V w; w.raw = __ldg(&ar[c].raw);
+      w.unpack(g);
+#pragma unroll
+      for (int q = 0; q < V::N; ++q) f[q] += g[q];
+    }
+#pragma unroll
+    for (int q = 0; q < V::N; ++q) { s_row[c * V::N + q] = f[q]; sum += f[q]; }
+  }
+  const float mean = block_sum(sum, red) / (float)D;
+  float sq = 0.f;
+  for (int c = threadIdx.x; c < D; c += kLnThreads) { const float d = s_row[c] - mean; sq = fmaf(d, d, sq); }
+  const float var = block_sum(sq, red) / (float)D;
+  const float rstd = 1.0f / sqrtf(var + eps);
+  const float* sh = shift + (long long)b * mod_ld;
+  const float* sc = scale + (long long)b * mod_ld;
+  V* out = reinterpret_cast<V*>(a + (long long)m * D);
+  for (int c = threadIdx.x; c < n_vec; c += kLnThreads) {
+    float f[V::N];
+#pragma unroll
+    for (int q = 0; q < V::N; ++q) {
+      const int col = c * V::N + q;
+      f[q] = fmaf((s_row[col] - mean) * rstd, 1.0f + sc[col], sh[col]);
+    }
+    V r; r.pack(f);
+    out[c] = r;
+  }
+}
+
+template <typename T>
+int extrapolate_t(const void* p, const void* l, void* o, long long n, float c, cudaStream_t s) {
+  extrapolate_kernel<T><<<stream_grid(n / Vec<T>::N), kStreamThreads, 0, s>>>((const T*)p, (const T*)l, (T*)o, n, c);
+  HERO_CUDA_TRY(cudaGetLastError());
+  return HERO_OK;
+}
+
+}  // namespace
+
+int launch_extrapolate(const void* g_prev, const void* g_last, void* out, long long n, int k, int d, int dtype,
+                       cudaStream_t s) {
+  const float c = (float)k / (float)d;
+  return dtype == HERO_DTYPE_BF16 ? extrapolate_t<__nv_bfloat16>(g_prev, g_last, out, n, c, s)
+                                  : extrapolate_t<float>(g_prev, g_last, out, n, c, s);
+}
+
+int launch_extrapolate_residual(void* x, const void* ga_prev, const void* ga_last, const void* gf_prev,
+                                const void* gf_last, long long n, int k, int d, int dtype, cudaStream_t s) {
+  const float c = (float)k / (float)d;
+  if (dtype == HERO_DTYPE_BF16) {
+    using T = __nv_bfloat16;
+    const long long n_vec = n / Vec<T>::N;
+    long long blocks = (n_vec + kStreamThreads - 1) / kStreamThreads;
+    blocks = blocks < 1 ? 1 : (blocks > (long long)num_sms() * 32 ? (long long)num_sms() * 32 : blocks);
+    extrapolate_residual_kernel<T><<<(int)blocks, kStreamThreads, 0, s>>>(
+        (T*)x, (const T*)ga_prev, (const T*)ga_last, (const T*)gf_prev, (const T*)gf_last, n, c);
+  } else {
+    using T = float;
+    const long long n_vec = n / Vec<T>::N;
+    long long blocks = (n_vec + kStreamThreads - 1) / kStreamThreads;
+    blocks = blocks < 1 ? 1 : (blocks > (long long)num_sms() * 32 ? (long long)num_sms() * 32 : blocks);
+    extrapolate_residual_kernel<T><<<(int)blocks, kStreamThreads, 0, s>>>(
+        (T*)x, (const T*)ga_prev, (const T*)ga_last, (const T*)gf_prev, (const T*)gf_last, n, c);
+  }
+  HERO_CUDA_TRY(cudaGetLastError());
+  return HERO_OK;
+}
+
+int launch_residual2(void* x, const void* ga, const void* gf, long long n, int dtype, cudaStream_t s) {
+  if (dtype == HERO_DTYPE_BF16) {
+    using T = __nv_bfloat16;
+    residual2_kernel<T><<<stream_grid(n / Vec<T>::N), kStreamThreads, 0, s>>>((T*)x, (const T*)ga, (const T*)gf, n);
+  } else {
+    residual2_kernel<float><<<stream_grid(n / 4), kStreamThreads, 0, s>>>((float*)x, (const float*)ga,
+                                                                           (const float*)gf, n);
+  }
+  HERO_CUDA_TRY(cudaGetLastError());
+  return HERO_OK;
+}
+
+static int move_rows(bool gather, const void* src, const int* idx, void* dst, int B, int N, int n_sel, int D,
+                     int dtype, cudaStream_t s) {
+  const long long row_bytes = (long long)D * dtype_size(dtype);
+  if (row_bytes % 16 != 0) return HERO_ERR_ALIGN;
+  const long long rows = (long long)B * n_sel;
+  if (rows == 0) return HERO_OK;
+  long long blocks = (rows + 7) / 8;   // 8 warps per CTA, one row per warp
+  const long long cap = (long long)num_sms() * 8;
+  if (blocks > cap) blocks = cap;
+  if (gather)
+    move_rows_kernel<true><<<(int)blocks, 256, 0, s>>>((const uint4*)src, idx, (uint4*)dst, B, N, n_sel,
+                                                       (int)(row_bytes / 16));
+  else
+    move_rows_kernel<false><<<(int)blocks, 256, 0, s>>>((const uint4*)src, idx, (uint4*)dst, B, N, n_sel,
+                                                        (int)(row_bytes / 16));
+  HERO_CUDA_TRY(cudaGetLastError());
+  return HERO_OK;
+}
+
+int launch_gather_rows(const void* src, const int* idx, void* dst, int B, int N, int n_sel, int D, int dtype,
+                       cudaStream_t s) {
+  return move_rows(true, src, idx, dst, B, N, n_sel, D, dtype, s);
+}
+int launch_scatter_rows(const void* src, const int* idx, void* dst, int B, int N, int n_sel, int D, int dtype,
+                        cudaStream_t s) {
+  return move_rows(false, src, idx, dst, B, N, n_sel, D, dtype, s);
+}
+
+int launch_modulation(const void* temb, const void* w_mod, const void* b_mod, float* mod, int B, int n_out, int E,
+                      int dtype, cudaStream_t s) {
+  if (B > kModMaxB) return HERO_ERR_ARG;
+  const size_t smem = (size_t)B * E * sizeof(float);
+  int blocks = (n_out + 7) / 8;
+  const int cap = num_sms() * 8;
+  if (blocks > cap) blocks = cap;
+  if (dtype == HERO_DTYPE_BF16) {
+    if (E % 8) return HERO_ERR_ALIGN;
+    modulation_kernel<__nv_bfloat16><<<blocks, 256, smem, s>>>((const __nv_bfloat16*)temb,
+                                                                (const __nv_bfloat16*)w_mod,
+                                                                (const __nv_bfloat16*)b_mod, mod, B, n_out, E);
+  } else {
+    if (E % 4) return HERO_ERR_ALIGN;
+    modulation_kernel<float><<<blocks, 256, smem, s>>>((const float*)temb, (const float*)w_mod,
+                                                       (const float*)b_mod, mod, B, n_out, E);
+  }
+  HERO_CUDA_TRY(cudaGetLastError());
+  return HERO_OK;
+}
+
+int launch_gather_ln_modulate(const void* x, const void* add, const int* idx, const float* shift,
+                              const float* scale, int mod_ld, void* a, int B, int N, int n_sel, int D, float eps,
+                              int dtype, cudaStream_t s) {
+  const long long rows = (long long)B * n_sel;
+  if (rows == 0) return HERO_OK;
+  const size_t smem = (size_t)D * sizeof(float);
+  if (dtype == HERO_DTYPE_BF16) {
+    using T = __nv_bfloat16;
+    if (D % 8) return HERO_ERR_ALIGN;
+    gather_ln_modulate_kernel<T><<<(unsigned)rows, kLnThreads, smem, s>>>((const T*)x, (const T*)add, idx, shift,
+                                                                           scale, mod_ld, (T*)a, N, n_sel, D, eps);
+  } else {
+    if (D % 4) return HERO_ERR_ALIGN;
+    gather_ln_modulate_kernel<float><<<(unsigned)rows, kLnThreads, smem, s>>>(
+        (const float*)x, (const float*)add, idx, shift, scale, mod_ld, (float*)a, N, n_sel, D, eps);
+  }
+  HERO_CUDA_TRY(cudaGetLastError());
+  return HERO_OK;
+}
+
+}  // namespace hero

@@ -1,0 +1,154 @@
+"""GPU parity, tensor-core kernels (tcgen05 + TMEM + TMA) through the C ABI against the float64
+oracle: the bf16 GEMM with its epilogues, flash attention over the full K/V, and whole bf16
+blocks (full pass, refresh, extrapolate) with teacher-forced caches."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import hero_oracle as O
+from workloads import synthetic as S
+from tests.util import make_pair, rel_l2, to_dev, to_host
+
+pytestmark = pytest.mark.gpu
+
+BF16_TOL = 2e-2          # rel-L2, bf16 GEMM/attention against the float64 oracle
+
+
+def H():
+    import paper_2508_17588_b200 as h
+    return h
+
+
+# ---------------------------------------------------------------- GEMM
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (1, 8, 8), (127, 264, 72), (300, 512, 256), (129, 3072, 3072),
+                                   (1000, 520, 1032), (4387, 768, 128)])
+@pytest.mark.parametrize("act", [0, 1])
+def test_gemm_matches_oracle(M, N, K, act):
+    rng = np.random.default_rng(M + N + K)
+    a = S.round_bf16(rng.standard_normal((M, K)).astype(np.float32))
+    w = S.round_bf16((rng.standard_normal((N, K)) * (1.0 / np.sqrt(K))).astype(np.float32))
+    bias = S.round_bf16(rng.standard_normal(N).astype(np.float32) * 0.1)
+    want = a.astype(np.float64) @ w.astype(np.float64).T + bias
+    if act:
+        want = O.gelu_tanh(want)
+    c = torch.full((M, N), float("nan"), device="cuda", dtype=torch.bfloat16)
+    H().hero_gemm_bf16(to_dev(a, "bf16"), to_dev(w, "bf16"), to_dev(bias, "bf16"), c, act)
+    H().hero_isolated_status()
+    got = to_host(c)
+    assert np.isfinite(got).all()
+    assert rel_l2(got, want) <= 5e-3          # one bf16 rounding of the output dominates
+    # element-wise: within one bf16 ulp of the exact value plus accumulation noise
+    assert np.abs(got - want).max() <= 2 ** -7 * np.abs(want).max() + 1e-3
+
+
+def test_gemm_many_tiles_per_cta():
+    """More tiles than SMs: every CTA walks several tiles and both TMEM accumulators."""
+    M, N, K = 2500, 3072, 192
+    rng = np.random.default_rng(7)
+    a = S.round_bf16(rng.standard_normal((M, K)).astype(np.float32))
+    w = S.round_bf16((rng.standard_normal((N, K)) / np.sqrt(K)).astype(np.float32))
+    bias = np.zeros(N, np.float32)
+    c = torch.empty((M, N), device="cuda", dtype=torch.bfloat16)
+    H().hero_gemm_bf16(to_dev(a, "bf16"), to_dev(w, "bf16"), to_dev(bias, "bf16"), c, 0)
+    H().hero_isolated_status()
+    want = a.astype(np.float64) @ w.astype(np.float64).T
+    assert rel_l2(to_host(c), want) <= 5e-3
+
+
+# ---------------------------------------------------------------- attention
+@pytest.mark.parametrize("B,n_q,N,heads", [(1, 128, 128, 1), (1, 1, 1, 1), (2, 37, 200, 2), (1, 130, 513, 3),
+                                           (2, 300, 1000, 2), (1, 64, 2300, 1)])
+def test_attention_matches_oracle(B, n_q, N, heads):
+    rng = np.random.default_rng(B * 7 + n_q + N)
+    D = heads * 64
+    q = S.round_bf16(rng.standard_normal((B, n_q, D)).astype(np.float32))
+    k = S.round_bf16(rng.standard_normal((B, N, D)).astype(np.float32))
+    v = S.round_bf16(rng.standard_normal((B, N, D)).astype(np.float32))
+    cfg = O.Config(n_blocks=1, n_shallow=1, hidden=D, n_heads=heads, head_dim=64, ffn_dim=8, temb_dim=8, batch=B,
+                   frames=1, grid_h=1, grid_w=1, n_text=0, patch_h=1, patch_w=1, ratio_num=1, ratio_den=1)
+    o = torch.full((B, n_q, D), float("nan"), device="cuda", dtype=torch.bfloat16)
+    H().hero_attention_bf16(to_dev(q, "bf16"), to_dev(k, "bf16"), to_dev(v, "bf16"), o, heads)
+    H().hero_isolated_status()
+    got = to_host(o)
+    assert np.isfinite(got).all()
+    for b in range(B):
+        want = O.attention(cfg, q[b].astype(np.float64), k[b].astype(np.float64), v[b].astype(np.float64))
+        assert rel_l2(got[b], want) <= 1e-2, b
+
+
+def test_attention_peaked_rows():
+    """Large logits: a query that matches one key must return that key's value row."""
+    rng = np.random.default_rng(11)
+    N, D = 700, 64
+    k = S.round_bf16(rng.standard_normal((1, N, D)).astype(np.float32))
+    v = S.round_bf16(rng.standard_normal((1, N, D)).astype(np.float32))
+    pick = np.array([0, 5, 127, 128, 400, 699])
+    q = S.round_bf16(30 * k[:, pick])
+    o = torch.empty((1, len(pick), D), device="cuda", dtype=torch.bfloat16)
+    H().hero_attention_bf16(to_dev(q, "bf16"), to_dev(k, "bf16"), to_dev(v, "bf16"), o, 1)
+    H().hero_isolated_status()
+    assert np.abs(to_host(o)[0] - v[0, pick]).max() <= 2e-2
+
+
+# ---------------------------------------------------------------- bf16 blocks
+SMALL_BF16 = dict(n_blocks=2, n_shallow=1, hidden=256, n_heads=4, head_dim=64, ffn_dim=768, temb_dim=64, batch=2,
+                  frames=3, grid_h=9, grid_w=11, n_text=10, patch_h=2, patch_w=2, ratio_num=1, ratio_den=4,
+                  quota_mode=0, warmup_full_steps=2, full_interval=3, dtype="bf16", has_gate=0, seed=21, steps=6)
+
+
+@pytest.mark.parametrize("gate", [0, 1])
+def test_bf16_small_model_steps_teacher_forced(gate):
+    """Full, refresh and extrapolate blocks in bf16 over 6 steps (full at 0, 1, 4).  Each step both
+    sides start from the same input; the oracle's caches are overwritten with the GPU's
+    bf16 caches after every step (teacher forcing) so the per-step error is what is graded."""
+    cfgd = dict(SMALL_BF16, has_gate=gate)
+    weights = [S.block_weights(cfgd, l) for l in range(cfgd["n_blocks"])]
+    for w in weights:        # larger modulation so that scale/shift/gate matter
+        w["w_mod"] = S.round_bf16(w["w_mod"] * 10)
+        w["b_mod"] = S.round_bf16(w["b_mod"] + (1.0 if gate else 0.0))
+    orc, hero, _ = make_pair(cfgd, weights)
+    x_host = S.tokens(cfgd)
+    for s in range(cfgd["steps"]):
+        temb = S.temb(cfgd, s)
+        want = orc.step(s, x_host, temb)
+        x = to_dev(x_host, "bf16")
+        hero.hero_step(s, x, to_dev(temb, "bf16"))
+        hero.hero_check_status()
+        err = rel_l2(to_host(x), want)
+        assert err <= BF16_TOL, (s, err)
+        assert np.array_equal(hero.hero_state_get(0, "ages").numpy(), orc.blocks[0].ages)
+        st = orc.blocks[0]
+        for name, ref in (("k", st.k_cache), ("v", st.v_cache), ("g_attn", st.g[0]), ("g_ffn", st.g[1])):
+            got = to_host(hero.hero_state_get(0, name))
+            assert rel_l2(got, ref) <= BF16_TOL, (s, name)
+            ref[...] = got                                   # teacher forcing
+        dp = orc.blocks[1]
+        for i, name in enumerate(("g_attn", "g_ffn")):
+            got = to_host(hero.hero_state_get(1, name))
+            assert rel_l2(got, dp.g_last[i]) <= BF16_TOL, (s, name)
+            dp.g_last[i][...] = got
+            if dp.g_prev[i] is not None:
+                gp = to_host(hero.hero_state_get(1, name + "_prev"))
+                assert rel_l2(gp, dp.g_prev[i]) <= BF16_TOL
+                dp.g_prev[i][...] = gp
+    hero.close()
+
+
+def test_bf16_refresh_keeps_unselected_rows_bit_identical():
+    cfgd = dict(SMALL_BF16, n_blocks=1, n_shallow=1)
+    _, hero, _ = make_pair(cfgd)
+    cfg = O.Config.from_dict(cfgd)
+    x = to_dev(S.tokens(cfgd), "bf16")
+    hero.hero_refresh_block(0, x, to_dev(S.temb(cfgd, 0), "bf16"))
+    before = {n: hero.hero_state_get(0, n).clone() for n in ("k", "v", "g_attn", "g_ffn")}
+    idx = torch.empty(cfg.n_video, dtype=torch.int32, device="cuda")
+    n = hero.hero_select_tokens(0, idx)
+    rows = idx[:n].cpu().numpy()
+    keep = np.setdiff1d(np.arange(cfg.n_rows), rows)
+    hero.hero_refresh_block(0, x, to_dev(S.temb(cfgd, 1), "bf16"), idx[:n])
+    hero.hero_check_status()
+    for name, b4 in before.items():
+        after = hero.hero_state_get(0, name)
+        assert torch.equal(after[:, keep], b4[:, keep]), name
+        assert not torch.equal(after[:, rows], b4[:, rows]), name
+    hero.close()
