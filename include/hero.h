@@ -107,6 +107,7 @@ int hero_next_n_sel(const hero_ctx *ctx, int block);
  * over the full cached K/V -> out-proj rows into G_attn -> x += G_attn -> LN+modulate ->
  * FFN (GELU-tanh) rows into G_ffn -> x += G_ffn.  d_idx == NULL with n_sel == N is the full
  * pass ("initial caching"): all rows, ages reset, deep blocks rotate their history slots.
+ * n_sel == 0 refreshes nothing and only adds the cached branches (d_idx is not read).
  * d_x [batch,N,hidden] is updated in place; d_temb is [batch, temb_dim]. */
 int hero_refresh_block(hero_ctx *ctx, int block, void *d_x, const void *d_temb,
                        const int *d_idx, int n_sel);

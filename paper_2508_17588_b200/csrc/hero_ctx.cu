@@ -355,15 +355,16 @@ int hero_refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, co
   if (!c || !d_x || !d_temb) return HERO_ERR_ARG;
   if (block < 0 || block >= c->cfg.n_blocks) return HERO_ERR_ARG;
   if (!aligned16(d_x) || !aligned16(d_temb)) return HERO_ERR_ALIGN;
+  if (n_sel == 0) {                                        // empty list: nothing refreshed,
+    if (block >= c->cfg.n_shallow) return HERO_ERR_ARG;    // the residual adds still happen
+    BlockMem& bm = c->blk[block];
+    return launch_residual2(d_x, bm.g[0], bm.g[1], c->elems, c->cfg.dtype, c->stream);
+  }
   if (d_idx == nullptr) {
     if (n_sel != c->N) return HERO_ERR_ARG;
   } else {
     if (n_sel < 0 || n_sel > c->N) return HERO_ERR_ARG;
     if (block >= c->cfg.n_shallow) return HERO_ERR_ARG;   // deep blocks keep no K/V cache to refresh against
-    if (n_sel == 0) {                                      // nothing refreshed: the residual adds still happen
-      BlockMem& bm = c->blk[block];
-      return launch_residual2(d_x, bm.g[0], bm.g[1], c->elems, c->cfg.dtype, c->stream);
-    }
   }
   return refresh_block(c, block, d_x, d_temb, d_idx, n_sel);
 }
