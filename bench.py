@@ -1,0 +1,378 @@
+#!/usr/bin/env python
+"""Benchmark of the HERO cached DiT step on B200.
+
+One "step" is one cached denoising step of the 42-block CogVideoX-5B-shaped DiT (config
+"dit42": 14 refresh blocks at 25 % + 28 extrapolated blocks, B=2 x N=17776 tokens, bf16):
+token selection, gather+LN, QKV/attention/out-proj/FFN on the refreshed rows with the merge
+into the caches, residual adds, and linear extrapolation in the deep blocks.  The two warm-up
+full steps that fill the caches are set-up, not timed; a full step is timed once and reported
+in `config` together with the 50-step schedule average.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl hero|reference] [--workload dit42|aether|tiny]
+
+Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank runs its own sequence on its
+own GPU (independent problems, no data-path collective): "scaling": "weak".
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from workloads import synthetic as S  # noqa: E402
+
+METRIC = "hero_cached_step_tokens_per_s"
+UNIT = "tokens/s"
+
+
+# --------------------------------------------------------------------------- helpers
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"],
+                    bf16_tflops_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons during the timed region (read-only queries)."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def refresh_flops(cfg, n_sel):
+    """Algorithmic flops of one refresh block on n = B*n_sel rows."""
+    B, D, F = cfg["batch"], cfg["hidden"], cfg["ffn_dim"]
+    N = S.n_rows(cfg)
+    n = B * n_sel
+    return dict(gemm=2 * n * D * 3 * D + 2 * n * D * D + 4 * n * D * F, attention=4 * n * N * D)
+
+
+# --------------------------------------------------------------------------- CPU baseline (oracle)
+class OracleSample:
+    """The CPU oracle, as it stands, on a bounded sample of one cached step, scaled to a whole
+    step.  Sample: one shallow block refreshed on its real selection with the K/V rewrite of every
+    selected row and the branch outputs of `sample_rows` of them, and one deep block's
+    extrapolation over the full tensor; a cached step is n_shallow times the first (outputs
+    scaled to all selected rows) plus n_deep times the second.  Caches hold synthetic values."""
+
+    def __init__(self, cfg):
+        from oracle import hero_oracle as O
+        self.cfg = cfg
+        one = dict(cfg, n_blocks=2, n_shallow=1)
+        w = [S.block_weights(one, 0)]
+        w.append(w[0])
+        self.orc = O.HeroOracle(O.Config.from_dict(one), w)
+        B, N, D = cfg["batch"], S.n_rows(cfg), cfg["hidden"]
+        rng = np.random.default_rng(0)
+        st = self.orc.blocks[0]
+        st.k_cache, st.v_cache = rng.standard_normal((B, N, D)), rng.standard_normal((B, N, D))
+        st.g = [rng.standard_normal((B, N, D)), rng.standard_normal((B, N, D))]
+        dp = self.orc.blocks[1]
+        dp.g_prev = [st.k_cache, st.v_cache]          # any full-size tensors do for timing
+        dp.g_last = [st.g[0], st.g[1]]
+        self.x = rng.standard_normal((B, N, D))
+        self.temb = S.temb(one, 2)
+
+    def step_seconds(self, sample_rows=256):
+        orc, cfg = self.orc, self.cfg
+        t0 = time.perf_counter()
+        rows = orc.select(0)
+        t_sel = time.perf_counter() - t0
+        sample_rows = min(sample_rows, len(rows))
+        small = max(sample_rows // 4, 1)
+        t0 = time.perf_counter()
+        orc.block_refresh(0, self.x, self.temb, rows, rows_out=rows[:sample_rows])
+        t_a = time.perf_counter() - t0
+        # the same with a quarter of the sample separates the fixed part from the per-row part
+        t0 = time.perf_counter()
+        orc.block_refresh(0, self.x, self.temb, rows, rows_out=rows[:small])
+        t_b = time.perf_counter() - t0
+        per_row = max(t_a - t_b, 0.0) / max(sample_rows - small, 1)
+        fixed = max(t_a - per_row * sample_rows, 0.0)
+        t_refresh = t_sel + fixed + per_row * len(rows)
+        t0 = time.perf_counter()
+        orc.block_extrapolate(1, self.x, 1, 5)
+        t_ext = time.perf_counter() - t0
+        n_sh, n_dp = cfg["n_shallow"], cfg["n_blocks"] - cfg["n_shallow"]
+        total = n_sh * t_refresh + n_dp * t_ext
+        detail = dict(select_s=t_sel, refresh_fixed_s=fixed, refresh_per_row_s=per_row, n_sel=int(len(rows)),
+                      extrapolate_block_s=t_ext, cpu_work_s=t_sel + t_a + t_b + t_ext)
+        return total, detail
+
+
+def cpu_cores_used():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max((p.get("num_threads", 1) for p in threadpool_info()), default=1)
+        return int(n)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args, cfg, rank, world):
+    """Reference arm: the oracle on this machine's host cores, on bounded samples of the same workload."""
+    if rank != 0:
+        return
+    tokens = cfg["batch"] * S.n_rows(cfg)
+    vals = []
+    sample_obj = OracleSample(cfg)
+    for i in range(args.warmup + args.steps):
+        sec, detail = sample_obj.step_seconds(sample_rows=128)
+        if i >= args.warmup:
+            vals.append(sec)
+    sec = statistics.mean(vals)
+    sample = ("per step: one shallow block refreshed on its 25 % selection (K/V of every selected row, branch "
+              "outputs of 128 rows, scaled to all) + one deep block extrapolated, scaled by block counts")
+    line = {"impl": "reference", "metric": METRIC, "value": tokens / sec, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "note": "oracle (numpy float64) timed on host cores"},
+            "cpu_baseline": {"value": tokens / sec, "unit": UNIT, "cores": cpu_cores_used(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": tokens / sec, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- CUDA arm
+def build_device_weights(cfg, device):
+    dt = torch.bfloat16 if cfg["dtype"] == "bf16" else torch.float32
+    weights = []
+    for l in range(cfg["n_blocks"]):
+        blk = {}
+        for name, shape in S.weight_shapes(cfg).items():
+            blk[name] = S.device_normal(cfg["seed"], name, shape, 0.02, l, None, device).to(dt).contiguous()
+        weights.append(blk)
+    return weights
+
+
+def run_hero(args, cfg, rank, world, local_rank):
+    import paper_2508_17588_b200 as H
+    H.load()                                     # fails loudly if the CUDA library is missing
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU path for the product arm")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    dt = torch.bfloat16 if cfg["dtype"] == "bf16" else torch.float32
+    run_cfg = dict(cfg, full_interval=0)         # after the two warm-up full steps every step is cached
+    run_cfg["seed"] = cfg["seed"] + rank         # each rank its own sequence (independent problems)
+    weights = build_device_weights(run_cfg, device)
+    hero = H.Hero(run_cfg, weights)
+    B, N, D = cfg["batch"], S.n_rows(cfg), cfg["hidden"]
+    tokens = B * N
+    x = S.device_normal(run_cfg["seed"], "x0", (B, N, D), 1.0, 0, None, device).to(dt)
+    tembs = [S.device_normal(run_cfg["seed"], "temb", (B, cfg["temb_dim"]), 1.0, s, None, device).to(dt)
+             for s in range(8)]
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    # set-up: the two "initial caching" full steps; the second one is timed for the record
+    hero.hero_step(0, x, tembs[0])
+    e0, e1 = ev(), ev()
+    torch.cuda.synchronize()
+    e0.record()
+    hero.hero_step(1, x, tembs[1])
+    e1.record()
+    torch.cuda.synchronize()
+    full_ms = e0.elapsed_time(e1)
+    hero.hero_check_status()
+
+    step = 2
+    for _ in range(args.warmup):
+        hero.hero_step(step, x, tembs[step % 8]); step += 1
+    torch.cuda.synchronize()
+    if dist:
+        dist.barrier()
+    sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else local_rank)
+    sampler.start()
+    launches0 = hero.hero_launch_count()
+    torch.cuda.synchronize()
+    e0, e1 = ev(), ev()
+    e0.record()
+    for _ in range(args.steps):
+        hero.hero_step(step, x, tembs[step % 8]); step += 1
+    e1.record()
+    torch.cuda.synchronize()
+    if dist:
+        dist.barrier()
+    total_ms = e0.elapsed_time(e1)
+    launches = hero.hero_launch_count() - launches0
+    clocks = sampler.stop()
+    hero.hero_check_status()
+    if dist:
+        t = torch.tensor([total_ms], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * tokens / (ms_per_step * 1e-3)
+
+    # per-category device time over two more cached steps (events around every launch)
+    n_prof = 2
+    hero.hero_profile_begin()
+    n_sel_seen = []
+    for _ in range(n_prof):
+        n_sel_seen.append(hero.hero_next_n_sel(0) if cfg["n_shallow"] else 0)
+        hero.hero_step(step, x, tembs[step % 8]); step += 1
+    prof = hero.hero_profile_end()
+    breakdown = {k: {"ms_per_step": v[0] / n_prof, "launches_per_step": v[1] / n_prof} for k, v in prof.items()}
+    peaks = measured_peaks()
+    roofline = None
+    if cfg["n_shallow"] and prof["attention"][1]:
+        n_sel = statistics.mean(n_sel_seen)
+        fl = refresh_flops(cfg, n_sel)
+        att_ms = prof["attention"][0] / prof["attention"][1]
+        gemm_ms_blk = prof["gemm"][0] / prof["attention"][1]          # four GEMMs per attention launch
+        achieved = fl["attention"] / (att_ms * 1e-3) / 1e12
+        peak = peaks["bf16_tflops_sustained"]
+        roofline = {"kernel": "tc_attention_kernel", "bound": "tensor", "achieved": achieved, "peak": peak,
+                    "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                    "peak_source": peaks["source"] + " (sustained cuBLAS bf16)",
+                    "flops_per_launch": fl["attention"], "ms_per_launch": att_ms,
+                    "gemm": {"achieved": fl["gemm"] / (gemm_ms_blk * 1e-3) / 1e12, "unit": "TFLOP/s",
+                             "frac": fl["gemm"] / (gemm_ms_blk * 1e-3) / 1e12 / peak,
+                             "flops_per_block": fl["gemm"], "ms_per_block": gemm_ms_blk}}
+        if breakdown["extrapolate"]["launches_per_step"]:
+            ext_ms = prof["extrapolate"][0] / prof["extrapolate"][1]
+            gbs = 6 * B * N * D * 2 / (ext_ms * 1e-3) / 1e9      # 5 reads + 1 write of [B,N,D] bf16
+            roofline["extrapolate"] = {"achieved": gbs, "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                                       "ms_per_launch": ext_ms}
+
+    # end to end through the host entry point: pinned host buffers, H2D + step + D2H per call
+    h_x = x.detach().cpu().pin_memory()
+    h_t = tembs[0].detach().cpu().pin_memory()
+    n_e2e = max(2, min(args.steps, 5))
+    hero.hero_step_host(step, h_x, h_t); step += 1
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(n_e2e):
+        hero.hero_step_host(step, h_x, h_t); step += 1
+    e2e_s = (time.perf_counter() - t0) / n_e2e
+    if dist:
+        t = torch.tensor([e2e_s], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    xb = h_x.numel() * h_x.element_size()
+    tb = h_t.numel() * h_t.element_size()
+    e2e = {"value": world * tokens / e2e_s, "unit": UNIT, "ms_per_step": e2e_s * 1e3,
+           "h2d_bytes_per_step": xb + tb, "d2h_bytes_per_step": xb}
+    hero.hero_check_status()
+    mem = hero.hero_device_bytes()
+    hero.close()
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        del weights
+        torch.cuda.empty_cache()
+        sec, detail = OracleSample(cfg).step_seconds(sample_rows=256)
+        cpu_baseline = {"value": tokens / sec, "unit": UNIT, "cores": cpu_cores_used(), "kind": "oracle",
+                        "sample": "one shallow block refreshed on its real selection (K/V of all selected rows, "
+                                  "branch outputs of 256 rows scaled to all) + one deep block extrapolated, scaled "
+                                  f"to {cfg['n_shallow']} + {cfg['n_blocks'] - cfg['n_shallow']} blocks; "
+                                  f"{detail['cpu_work_s']:.1f} s of CPU work",
+                        "ms_per_step": sec * 1e3}
+
+    if rank == 0:
+        n_full = sum(1 for s in range(cfg["steps"])
+                     if s < cfg["warmup_full_steps"] or
+                     (cfg["full_interval"] > 0 and (s - (cfg["warmup_full_steps"] - 1)) % cfg["full_interval"] == 0))
+        sched_ms = (n_full * full_ms + (cfg["steps"] - n_full) * ms_per_step) / cfg["steps"]
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": cfg["dtype"], "data": "synthetic",
+                "config": {"workload": args.workload, "blocks": cfg["n_blocks"], "refresh_blocks": cfg["n_shallow"],
+                           "refresh_ratio": cfg["ratio_num"] / cfg["ratio_den"], "batch": B, "tokens_per_seq": N,
+                           "hidden": D, "l2": "inputs larger than L2 (each step streams > 30 GB of caches)",
+                           "full_step_ms": full_ms, "schedule_avg_ms_per_step": sched_ms,
+                           "schedule": "%d full + %d cached of %d steps" % (n_full, cfg["steps"] - n_full, cfg["steps"]),
+                           "device_bytes": mem, "parallelism": "replicas" if world > 1 else "single"},
+                "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "breakdown_ms": breakdown}
+        if roofline:
+            line["roofline"] = roofline
+        if cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline
+        print(json.dumps(line))
+    if dist:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="hero", choices=["hero", "reference"])
+    ap.add_argument("--workload", default="dit42", choices=["dit42", "aether", "tiny"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    cfg = dict(S.CONFIGS[args.workload])
+    if args.impl == "reference":
+        run_reference(args, cfg, rank, world)
+    else:
+        run_hero(args, cfg, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

@@ -90,6 +90,23 @@ const char *hero_last_cuda_error(void);
 /* Bytes of device memory the context allocated. */
 long long hero_device_bytes(const hero_ctx *ctx);
 
+/* Kernel launches enqueued by this context since hero_init (all categories). */
+long long hero_launch_count(const hero_ctx *ctx);
+
+/* Per-category device timing.  Between hero_profile_begin and hero_profile_end every kernel the
+ * context launches is bracketed by CUDA events on its stream; hero_profile_end synchronises and
+ * fills ms[HERO_PROF_CATEGORIES] (summed event time) and launches[HERO_PROF_CATEGORIES]. */
+#define HERO_PROF_SELECT      0   /* token selection */
+#define HERO_PROF_MODULATION  1   /* adaLN vectors from the timestep embedding */
+#define HERO_PROF_GATHER_LN   2   /* gather + LayerNorm + modulate */
+#define HERO_PROF_GEMM        3   /* QKV, out-proj, FFN up/down (epilogue scatters into the caches) */
+#define HERO_PROF_ATTENTION   4   /* refreshed queries over the full cached K/V */
+#define HERO_PROF_RESIDUAL    5   /* x += G_attn + G_ffn, all rows */
+#define HERO_PROF_EXTRAPOLATE 6   /* Eq. 5 + residual add in deep blocks */
+#define HERO_PROF_CATEGORIES  7
+int hero_profile_begin(hero_ctx *ctx);
+int hero_profile_end(hero_ctx *ctx, double *h_ms, long long *h_launches);
+
 /* ---- the method's calls (Algorithm 1) ------------------------------------ */
 
 /* S(z) of Eq. 4 for one shallow block: per patch take the quota's worth of tokens with the

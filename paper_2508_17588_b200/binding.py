@@ -18,9 +18,11 @@ OK, ERR_ARG, ERR_ALIGN, ERR_CAP, ERR_STATE, ERR_CUDA, ERR_TIMEOUT, ERR_NOMEM = 0
 DTYPE_FP32, DTYPE_BF16 = 0, 1
 STATE = dict(ages=0, calls=1, k=2, v=3, g_attn=4, g_ffn=5, g_attn_prev=6, g_ffn_prev=7, steps=8)
 
+PROF_CATEGORIES = ("select", "modulation", "gather_ln", "gemm", "attention", "residual", "extrapolate")
+
 EXPORTS = [
     "hero_init", "hero_reset", "hero_destroy", "hero_strerror", "hero_check_status", "hero_last_cuda_error",
-    "hero_device_bytes", "hero_select_tokens", "hero_next_n_sel", "hero_refresh_block",
+    "hero_device_bytes", "hero_launch_count", "hero_profile_begin", "hero_profile_end", "hero_select_tokens", "hero_next_n_sel", "hero_refresh_block",
     "hero_extrapolate_block", "hero_step", "hero_step_host", "hero_is_full_step", "hero_extrapolate",
     "hero_gather_rows", "hero_scatter_rows", "hero_gemm_bf16", "hero_attention_bf16", "hero_isolated_status",
     "hero_state_get", "hero_state_set",
@@ -70,6 +72,9 @@ def load() -> C.CDLL:
         "hero_check_status": (i, [vp]),
         "hero_last_cuda_error": (C.c_char_p, []),
         "hero_device_bytes": (ll, [vp]),
+        "hero_launch_count": (ll, [vp]),
+        "hero_profile_begin": (i, [vp]),
+        "hero_profile_end": (i, [vp, C.POINTER(C.c_double), C.POINTER(ll)]),
         "hero_select_tokens": (i, [vp, i, vp, i, ip]),
         "hero_next_n_sel": (i, [vp, i]),
         "hero_refresh_block": (i, [vp, i, vp, vp, vp, i]),
@@ -203,6 +208,19 @@ class Hero:
 
     def hero_device_bytes(self) -> int:
         return self.lib.hero_device_bytes(self.ctx)
+
+    def hero_launch_count(self) -> int:
+        return self.lib.hero_launch_count(self.ctx)
+
+    def hero_profile_begin(self):
+        _check(self.lib.hero_profile_begin(self.ctx), "hero_profile_begin")
+
+    def hero_profile_end(self) -> dict:
+        """{category: (summed device ms, launches)} since hero_profile_begin."""
+        ms = (C.c_double * len(PROF_CATEGORIES))()
+        n = (C.c_longlong * len(PROF_CATEGORIES))()
+        _check(self.lib.hero_profile_end(self.ctx, ms, n), "hero_profile_end")
+        return {name: (ms[i], n[i]) for i, name in enumerate(PROF_CATEGORIES)}
 
     # ---- state access ---------------------------------------------------------
     def _state_tensor(self, what: str) -> torch.Tensor:

@@ -51,9 +51,38 @@ struct hero_ctx {
   int mode1_n_sel = 0;
   long long bytes = 0;
   std::vector<void*> allocs;
+  // launch accounting and optional per-category event timing
+  long long launches[HERO_PROF_CATEGORIES] = {0};
+  bool profiling = false;
+  struct ProfSpan { int cat; cudaEvent_t a, b; };
+  std::vector<ProfSpan> spans;        // recorded since hero_profile_begin
+  std::vector<ProfSpan> span_pool;    // reusable event pairs
 };
 
 namespace {
+
+// Every kernel launch goes through this: counts it and, while profiling, brackets it with events.
+struct LaunchScope {
+  hero_ctx* c; int cat; cudaEvent_t stop = nullptr;
+  LaunchScope(hero_ctx* ctx, int category) : c(ctx), cat(category) {
+    c->launches[cat]++;
+    if (!c->profiling) return;
+    hero_ctx::ProfSpan sp;
+    if (!c->span_pool.empty()) { sp = c->span_pool.back(); c->span_pool.pop_back(); }
+    else if (cudaEventCreate(&sp.a) != cudaSuccess || cudaEventCreate(&sp.b) != cudaSuccess) return;
+    sp.cat = cat;
+    cudaEventRecord(sp.a, c->stream);
+    stop = sp.b;
+    c->spans.push_back(sp);
+  }
+  ~LaunchScope() { if (stop) cudaEventRecord(stop, c->stream); }
+};
+#define HERO_LAUNCH(ctx, cat, expr)        \
+  do {                                     \
+    LaunchScope scope__(ctx, cat);         \
+    int r__ = (expr);                      \
+    if (r__ != HERO_OK) return r__;        \
+  } while (0)
 
 int dev_alloc(hero_ctx* c, void** p, size_t bytes) {
   *p = nullptr;
@@ -107,12 +136,14 @@ bool is_full(const hero_config& g, int step) {
 }
 
 int run_gemm(hero_ctx* c, const void* a, const void* w, const void* bias, int M, int Nout, int K, const GemmOut& out) {
+  LaunchScope scope(c, HERO_PROF_GEMM);
   if (c->cfg.dtype == HERO_DTYPE_BF16) return launch_tc_gemm(a, w, bias, M, Nout, K, out, c->d_status, c->stream);
   return launch_simt_gemm(a, w, bias, M, Nout, K, out, c->cfg.dtype, c->stream);
 }
 
 int run_attention(hero_ctx* c, const void* q, const void* k, const void* v, void* o, int n_q) {
   const hero_config& g = c->cfg;
+  LaunchScope scope(c, HERO_PROF_ATTENTION);
   if (g.dtype == HERO_DTYPE_BF16)
     return launch_tc_attention(q, k, v, o, g.batch, n_q, c->N, g.n_heads, c->d_status, c->stream);
   return launch_simt_attention(q, k, v, o, g.batch, n_q, c->N, g.n_heads, g.head_dim, g.dtype, c->stream);
@@ -139,7 +170,8 @@ int refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, const i
     kdst = bm.k; vdst = bm.v; ga = bm.g[0]; gf = bm.g[1];
   }
 
-  HERO_TRY(launch_modulation(d_temb, w.w_mod, w.b_mod, c->mod, B, mod_ld, g.temb_dim, g.dtype, c->stream));
+  HERO_LAUNCH(c, HERO_PROF_MODULATION,
+              launch_modulation(d_temb, w.w_mod, w.b_mod, c->mod, B, mod_ld, g.temb_dim, g.dtype, c->stream));
   const float* shift1 = c->mod;
   const float* scale1 = c->mod + D;
   const float* shift2 = c->mod + 2 * D;
@@ -148,8 +180,9 @@ int refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, const i
   const float* gate2 = g.has_gate ? c->mod + 5 * D : nullptr;
 
   // attention branch
-  HERO_TRY(launch_gather_ln_modulate(d_x, nullptr, d_idx, shift1, scale1, mod_ld, c->ws_a, B, N, n_sel, D, 1e-5f,
-                                     g.dtype, c->stream));
+  HERO_LAUNCH(c, HERO_PROF_GATHER_LN,
+              launch_gather_ln_modulate(d_x, nullptr, d_idx, shift1, scale1, mod_ld, c->ws_a, B, N, n_sel, D, 1e-5f,
+                                        g.dtype, c->stream));
   GemmOut o_qkv = {};
   o_qkv.ptr[0] = c->ws_q; o_qkv.ld[0] = D; o_qkv.scatter[0] = 0;
   o_qkv.ptr[1] = kdst;    o_qkv.ld[1] = D; o_qkv.scatter[1] = 1;
@@ -164,8 +197,9 @@ int refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, const i
   HERO_TRY(run_gemm(c, c->ws_o, w.w_o, w.b_o, M, D, D, o_attn));
 
   // FFN branch: its input rows are x + G_attn (the residual add is applied to x once, below)
-  HERO_TRY(launch_gather_ln_modulate(d_x, ga, d_idx, shift2, scale2, mod_ld, c->ws_a, B, N, n_sel, D, 1e-5f,
-                                     g.dtype, c->stream));
+  HERO_LAUNCH(c, HERO_PROF_GATHER_LN,
+              launch_gather_ln_modulate(d_x, ga, d_idx, shift2, scale2, mod_ld, c->ws_a, B, N, n_sel, D, 1e-5f,
+                                        g.dtype, c->stream));
   GemmOut o_up = {};
   o_up.ptr[0] = c->ws_u; o_up.ld[0] = F; o_up.scatter[0] = 0;
   o_up.seg_cols = F; o_up.idx = d_idx; o_up.n_sel = n_sel; o_up.n_rows = N; o_up.act = 1;
@@ -177,7 +211,7 @@ int refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, const i
   HERO_TRY(run_gemm(c, c->ws_u, w.w_2, w.b_2, M, D, F, o_dn));
 
   // x = (x + G_attn) + G_ffn for every row: fresh rows and cached rows alike
-  HERO_TRY(launch_residual2(d_x, ga, gf, c->elems, g.dtype, c->stream));
+  HERO_LAUNCH(c, HERO_PROF_RESIDUAL, launch_residual2(d_x, ga, gf, c->elems, g.dtype, c->stream));
 
   if (full) {
     if (deep) {
@@ -194,8 +228,10 @@ int extrapolate_block(hero_ctx* c, int block, void* d_x, int k, int d) {
   BlockMem& bm = c->blk[block];
   if (bm.n_hist == 0) return HERO_ERR_STATE;
   const int last = bm.last_slot, prev = bm.n_hist >= 2 ? (last ^ 1) : last;   // one slot only: Delta = 0
-  return launch_extrapolate_residual(d_x, bm.hist[0][prev], bm.hist[0][last], bm.hist[1][prev], bm.hist[1][last],
-                                     c->elems, k, d, c->cfg.dtype, c->stream);
+  HERO_LAUNCH(c, HERO_PROF_EXTRAPOLATE,
+              launch_extrapolate_residual(d_x, bm.hist[0][prev], bm.hist[0][last], bm.hist[1][prev],
+                                          bm.hist[1][last], c->elems, k, d, c->cfg.dtype, c->stream));
+  return HERO_OK;
 }
 
 int validate(const hero_config* g) {
@@ -244,6 +280,8 @@ void hero_destroy(hero_ctx* c) {
   if (!c) return;
   if (c->stream) cudaStreamSynchronize(c->stream); else cudaDeviceSynchronize();
   for (void* p : c->allocs) cudaFree(p);
+  for (auto& sp : c->spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
+  for (auto& sp : c->span_pool) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
   delete c;
 }
 
@@ -316,6 +354,37 @@ int hero_reset(hero_ctx* c) {
 
 long long hero_device_bytes(const hero_ctx* c) { return c ? c->bytes : 0; }
 
+long long hero_launch_count(const hero_ctx* c) {
+  if (!c) return 0;
+  long long n = 0;
+  for (int i = 0; i < HERO_PROF_CATEGORIES; ++i) n += c->launches[i];
+  return n;
+}
+
+int hero_profile_begin(hero_ctx* c) {
+  if (!c) return HERO_ERR_ARG;
+  for (auto& sp : c->spans) c->span_pool.push_back(sp);
+  c->spans.clear();
+  c->profiling = true;
+  return HERO_OK;
+}
+
+int hero_profile_end(hero_ctx* c, double* ms, long long* launches) {
+  if (!c || !ms || !launches) return HERO_ERR_ARG;
+  c->profiling = false;
+  HERO_CUDA_TRY(cudaStreamSynchronize(c->stream));
+  for (int i = 0; i < HERO_PROF_CATEGORIES; ++i) { ms[i] = 0.0; launches[i] = 0; }
+  for (auto& sp : c->spans) {
+    float t = 0.f;
+    HERO_CUDA_TRY(cudaEventElapsedTime(&t, sp.a, sp.b));
+    ms[sp.cat] += t;
+    launches[sp.cat]++;
+    c->span_pool.push_back(sp);
+  }
+  c->spans.clear();
+  return HERO_OK;
+}
+
 int hero_check_status(hero_ctx* c) {
   if (!c) return HERO_ERR_ARG;
   int st[4] = {0, 0, 0, 0};
@@ -344,7 +413,7 @@ int hero_select_tokens(hero_ctx* c, int block, int* d_idx, int cap, int* n_sel) 
   batch.block[0] = block; batch.call[0] = bm.calls;
   batch.ages_in[0] = bm.ages[bm.ages_cur]; batch.ages_out[0] = bm.ages[bm.ages_cur ^ 1];
   batch.idx[0] = d_idx;
-  HERO_TRY(launch_select(geom_of(c->cfg), batch, c->stream));
+  HERO_LAUNCH(c, HERO_PROF_SELECT, launch_select(geom_of(c->cfg), batch, c->stream));
   bm.ages_cur ^= 1;
   bm.calls++;
   if (n_sel) *n_sel = n;
@@ -358,7 +427,8 @@ int hero_refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, co
   if (n_sel == 0) {                                        // empty list: nothing refreshed,
     if (block >= c->cfg.n_shallow) return HERO_ERR_ARG;    // the residual adds still happen
     BlockMem& bm = c->blk[block];
-    return launch_residual2(d_x, bm.g[0], bm.g[1], c->elems, c->cfg.dtype, c->stream);
+    HERO_LAUNCH(c, HERO_PROF_RESIDUAL, launch_residual2(d_x, bm.g[0], bm.g[1], c->elems, c->cfg.dtype, c->stream));
+    return HERO_OK;
   }
   if (d_idx == nullptr) {
     if (n_sel != c->N) return HERO_ERR_ARG;
@@ -407,7 +477,7 @@ int hero_step(hero_ctx* c, int step, void* d_x, const void* d_temb) {
       batch.ages_in[l] = bm.ages[bm.ages_cur]; batch.ages_out[l] = bm.ages[bm.ages_cur ^ 1];
       batch.idx[l] = c->idx_ws + (size_t)l * c->idx_cap;
     }
-    HERO_TRY(launch_select(geom_of(g), batch, c->stream));
+    HERO_LAUNCH(c, HERO_PROF_SELECT, launch_select(geom_of(g), batch, c->stream));
     for (int l = 0; l < g.n_shallow; ++l) { c->blk[l].ages_cur ^= 1; c->blk[l].calls++; }
   }
   for (int l = 0; l < g.n_blocks; ++l) {
@@ -415,7 +485,8 @@ int hero_step(hero_ctx* c, int step, void* d_x, const void* d_temb) {
       if (n_sel[l] > 0) {
         HERO_TRY(refresh_block(c, l, d_x, d_temb, c->idx_ws + (size_t)l * c->idx_cap, n_sel[l]));
       } else {
-        HERO_TRY(launch_residual2(d_x, c->blk[l].g[0], c->blk[l].g[1], c->elems, g.dtype, c->stream));
+        HERO_LAUNCH(c, HERO_PROF_RESIDUAL,
+                    launch_residual2(d_x, c->blk[l].g[0], c->blk[l].g[1], c->elems, g.dtype, c->stream));
       }
     } else {
       HERO_TRY(extrapolate_block(c, l, d_x, k, d));
