@@ -8,7 +8,7 @@ into the caches, residual adds, and linear extrapolation in the deep blocks.  Th
 full steps that fill the caches are set-up, not timed; a full step is timed once and reported
 in `config` together with the 50-step schedule average.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl hero|reference] [--workload dit42|aether|tiny]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl hero|reference] [--workload dit42|aether|tiny|kernels [--only LIST] [--small]]
 
 Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank runs its own sequence on its
 own GPU (independent problems, no data-path collective): "scaling": "weak".
@@ -355,18 +355,157 @@ def run_hero(args, cfg, rank, world, local_rank):
         dist.destroy_process_group()
 
 
+# --------------------------------------------------------------------------- isolated kernels
+def _time_flushed(fn, iters, warmup, flush):
+    """Median device time (ms) of fn() with L2 flushed (a write larger than L2) before each call."""
+    ts = []
+    for i in range(warmup + iters):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        e1.synchronize()
+        if i >= warmup:
+            ts.append(e0.elapsed_time(e1))
+    return statistics.median(ts)
+
+
+def run_kernels(args):
+    """Each kernel of the cached step alone, at the shapes of the isolated-kernel and one-block
+    workloads ([2, 17776, 3072] bf16, index lists at 10/25/50 %), against its own roofline.
+    `--small` shrinks the tensor-core cases to what a profiler capture handles in seconds."""
+    import paper_2508_17588_b200 as H
+    H.load()
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU path for the product arm")
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    peaks = measured_peaks()
+    cfg = dict(S.CONFIGS["kernels"])
+    B, N, D, F = cfg["batch"], S.n_rows(cfg), cfg["hidden"], cfg["ffn_dim"]
+    heads = cfg["n_heads"]
+    only = set(args.only.split(",")) if args.only else None
+    want = lambda name: only is None or name in only
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    iters, warm = max(args.steps, 5), max(args.warmup, 3)
+    bf = torch.bfloat16
+    out = {}
+
+    def rnd(*shape, std=1.0):
+        return (torch.randn(*shape, device=dev) * std).to(bf)
+
+    def hbm(name, ms, nbytes, **extra):
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        out[name] = dict(ms=ms, bytes=nbytes, achieved=gbs, unit="GB/s", frac=gbs / peaks["hbm_gbs"],
+                         frac_of_8tbs=gbs / 8000.0, bound="hbm", **extra)
+
+    def tensor(name, ms, flops, **extra):
+        tf = flops / (ms * 1e-3) / 1e12
+        out[name] = dict(ms=ms, flops=flops, achieved=tf, unit="TFLOP/s", frac=tf / peaks["bf16_tflops"],
+                         frac_of_sustained=tf / peaks["bf16_tflops_sustained"], frac_of_2250=tf / 2250.0,
+                         bound="tensor", **extra)
+
+    # index lists from the library's own sampler (a context with a one-head block: only geometry matters)
+    lists = {}
+    if want("gather") or want("scatter") or want("select"):
+        small_cfg = dict(cfg, hidden=64, n_heads=1, ffn_dim=64, temb_dim=64, n_blocks=1, n_shallow=1)
+        w = [{k: torch.zeros(s, device=dev, dtype=bf) for k, s in S.weight_shapes(small_cfg).items()}]
+        for num, den in ((1, 10), (1, 4), (1, 2)):
+            hero = H.Hero(dict(small_cfg, ratio_num=num, ratio_den=den), w)
+            idx = torch.empty(S.n_video(cfg), dtype=torch.int32, device=dev)
+            n = hero.hero_select_tokens(0, idx)
+            lists[f"{num}/{den}"] = idx[:n].clone()
+            if want("select") and (num, den) == (1, 4):
+                ms = _time_flushed(lambda: hero.hero_select_tokens(0, idx), iters, warm, flush)
+                out["select_25"] = dict(ms=ms, tokens=S.n_video(cfg), bound="latency",
+                                        note="integer work on 35 KB of counters; no bandwidth figure applies")
+            hero.close()
+
+    if want("extrapolate"):
+        a, b_, o = rnd(B, N, D), rnd(B, N, D), torch.empty(B, N, D, device=dev, dtype=bf)
+        ms = _time_flushed(lambda: H.hero_extrapolate(a, b_, o, 4, 5), iters, warm, flush)
+        hbm("extrapolate", ms, 3 * a.numel() * 2)
+        del a, b_, o
+    if want("gather") or want("scatter"):
+        src = rnd(B, N, D)
+        for key, idx in lists.items():
+            comp = torch.empty(B, idx.numel(), D, device=dev, dtype=bf)
+            nbytes = 2 * B * idx.numel() * D * 2 + 4 * idx.numel()
+            if want("gather"):
+                hbm(f"gather_{key}", _time_flushed(lambda: H.hero_gather_rows(src, idx, comp), iters, warm, flush),
+                    nbytes, rows=idx.numel())
+            if want("scatter"):
+                hbm(f"scatter_{key}", _time_flushed(lambda: H.hero_scatter_rows(comp, idx, src), iters, warm, flush),
+                    nbytes, rows=idx.numel())
+        del src
+    if want("attention"):
+        cases = [(1, 768)] if args.small else [(B, 1755), (B, 4387), (B, 8775)]
+        for bb, nq in cases:
+            q, k, v = rnd(bb, nq, D), rnd(bb, N, D), rnd(bb, N, D)
+            o = torch.empty_like(q)
+            ms = _time_flushed(lambda: H.hero_attention_bf16(q, k, v, o, heads), iters, warm, flush)
+            H.hero_isolated_status()
+            tensor(f"attention_b{bb}_q{nq}", ms, 4 * bb * nq * N * D)
+            del q, k, v, o
+    if want("gemm"):
+        M = 2048 if args.small else B * 4387
+        shapes = [("qkv", 3 * D, D, 0)] if args.small else [("qkv", 3 * D, D, 0), ("out", D, D, 0),
+                                                             ("ffn_up", F, D, 1), ("ffn_down", D, F, 0)]
+        for name, n_out, kk, act in shapes:
+            a, w_, bias = rnd(M, kk), rnd(n_out, kk, std=0.02), rnd(n_out, std=0.02)
+            c = torch.empty(M, n_out, device=dev, dtype=bf)
+            ms = _time_flushed(lambda: H.hero_gemm_bf16(a, w_, bias, c, act), iters, warm, flush)
+            H.hero_isolated_status()
+            tensor(f"gemm_{name}_m{M}", ms, 2 * M * n_out * kk)
+            del a, w_, bias, c
+    if want("block") and not args.small:
+        bcfg = dict(S.CONFIGS["block"])
+        weights = build_device_weights(bcfg, dev)
+        x = S.device_normal(bcfg["seed"], "x0", (B, N, D), 1.0, 0, None, dev).to(bf)
+        temb = S.device_normal(bcfg["seed"], "temb", (B, bcfg["temb_dim"]), 1.0, 0, None, dev).to(bf)
+        for num, den in ((1, 10), (1, 4), (1, 2), (1, 1)):
+            hero = H.Hero(dict(bcfg, ratio_num=num, ratio_den=den), weights)
+            hero.hero_refresh_block(0, x, temb)                 # fill the caches (full pass)
+            idx = torch.empty(S.n_video(bcfg), dtype=torch.int32, device=dev)
+            state = {}
+
+            def one():
+                if (num, den) == (1, 1):
+                    state["n"] = N
+                    hero.hero_refresh_block(0, x, temb)
+                else:
+                    state["n"] = hero.hero_select_tokens(0, idx)
+                    hero.hero_refresh_block(0, x, temb, idx, state["n"])
+            ms = _time_flushed(one, iters, warm, flush)
+            hero.hero_check_status()
+            fl = refresh_flops(bcfg, state["n"])
+            tensor(f"refresh_block_{num}/{den}", ms, fl["gemm"] + fl["attention"], n_sel=state["n"])
+            hero.close()
+    print(json.dumps({"workload": "kernels", "small": bool(args.small), "iters": iters, "timing":
+                      "CUDA events, median, L2 flushed by a 256 MiB write before every call",
+                      "peaks": peaks, "kernels": out}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="hero", choices=["hero", "reference"])
-    ap.add_argument("--workload", default="dit42", choices=["dit42", "aether", "tiny"])
+    ap.add_argument("--workload", default="dit42", choices=["dit42", "aether", "tiny", "kernels"])
+    ap.add_argument("--only", default="", help="kernels workload: comma list of select,extrapolate,gather,scatter,"
+                                               "attention,gemm,block")
+    ap.add_argument("--small", action="store_true", help="kernels workload: profiler-sized tensor-core cases")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.workload == "kernels" and args.impl == "hero":
+        if rank == 0:
+            run_kernels(args)
+        return
     cfg = dict(S.CONFIGS[args.workload])
     if args.impl == "reference":
         run_reference(args, cfg, rank, world)
