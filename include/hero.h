@@ -163,6 +163,27 @@ int hero_gemm_bf16(const void *d_a, const void *d_w, const void *d_bias, void *d
 int hero_attention_bf16(const void *d_q, const void *d_k, const void *d_v, void *d_o,
                         int B, int n_q, int N, int heads, void *stream);
 
+/* hero_attention_bf16 without any allocation (the paper has no counterpart: this entry point
+ * exists for the sake of callers, not of the method).  hero_attention_bf16 obtains its status
+ * word with cudaMalloc on first use; a caller that must never enter the CUDA allocator - a
+ * serving loop that cannot take the device-wide synchronisation cudaMalloc/cudaFree imply, a
+ * process whose framework already owns all device memory, code running where allocation is
+ * forbidden - calls this instead.  Same arguments and same result (bit for bit); its scratch is
+ * a fixed 64.25 KiB array inside the library image, present on every GPU that loads the library
+ * until the process exits.
+ *   - Limit: ceil(n_q / 256) * heads * B <= 16384 (one scratch word per thread block); beyond
+ *     that nothing is launched, HERO_ERR_CAP is returned and hero_last_cuda_error() says why.
+ *   - The first call on each device resolves the array's device address and sets the kernel's
+ *     shared-memory limit (no allocation either); make that call before any stream capture.
+ *   - Every call reuses the one array and clears the words it needs on `stream` before the
+ *     kernel; calls that overlap on the GPU race on it, so order them on one stream or with events.
+ *   - h_gave_up (host, may be NULL): when given, the call synchronises `stream`, stores the number
+ *     of thread blocks that gave up on a bounded device-side wait (0 in a healthy run) and
+ *     returns HERO_ERR_TIMEOUT if it is not 0.  When NULL the call stays asynchronous.
+ * Calls cudaMalloc, cudaFree or any allocating library routine: never. */
+int hero_attention_bf16_static(const void *d_q, const void *d_k, const void *d_v, void *d_o,
+                               int B, int n_q, int N, int heads, void *stream, int *h_gave_up);
+
 /* Synchronise `stream` and return HERO_ERR_TIMEOUT if hero_gemm_bf16 / hero_attention_bf16 gave
  * up on a bounded device-side wait since the last poll, else HERO_OK. */
 int hero_isolated_status(void *stream);

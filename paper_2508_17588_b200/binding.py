@@ -24,7 +24,7 @@ EXPORTS = [
     "hero_init", "hero_reset", "hero_destroy", "hero_strerror", "hero_check_status", "hero_last_cuda_error",
     "hero_device_bytes", "hero_launch_count", "hero_profile_begin", "hero_profile_end", "hero_select_tokens", "hero_next_n_sel", "hero_refresh_block",
     "hero_extrapolate_block", "hero_step", "hero_step_host", "hero_is_full_step", "hero_extrapolate",
-    "hero_gather_rows", "hero_scatter_rows", "hero_gemm_bf16", "hero_attention_bf16", "hero_isolated_status",
+    "hero_gather_rows", "hero_scatter_rows", "hero_gemm_bf16", "hero_attention_bf16", "hero_attention_bf16_static", "hero_isolated_status",
     "hero_state_get", "hero_state_set",
 ]
 
@@ -87,6 +87,7 @@ def load() -> C.CDLL:
         "hero_scatter_rows": (i, [vp, vp, vp, i, i, i, i, i, vp]),
         "hero_gemm_bf16": (i, [vp, vp, vp, vp, i, i, i, i, vp]),
         "hero_attention_bf16": (i, [vp, vp, vp, vp, i, i, i, i, vp]),
+        "hero_attention_bf16_static": (i, [vp, vp, vp, vp, i, i, i, i, vp, ip]),
         "hero_isolated_status": (i, [vp]),
         "hero_state_get": (i, [vp, i, i, vp, ll]),
         "hero_state_set": (i, [vp, i, i, vp, ll]),
@@ -284,6 +285,19 @@ def hero_attention_bf16(q, k, v, o, heads: int):
     N = k.shape[1]
     _check(load().hero_attention_bf16(_ptr(q), _ptr(k), _ptr(v), _ptr(o), B, n_q, N, heads, _stream()),
            "hero_attention_bf16")
+    return o
+
+
+def hero_attention_bf16_static(q, k, v, o, heads: int, check: bool = True):
+    """hero_attention_bf16 for callers that must not allocate device memory: the kernel's scratch is a
+    fixed array inside the library.  With check=True the call waits for the result and raises if any
+    thread block gave up on a bounded wait; with check=False it only enqueues the work."""
+    _require_cuda()
+    B, n_q, _ = q.shape
+    N = k.shape[1]
+    gave_up = C.c_int(0)
+    _check(load().hero_attention_bf16_static(_ptr(q), _ptr(k), _ptr(v), _ptr(o), B, n_q, N, heads, _stream(),
+                                             C.byref(gave_up) if check else None), "hero_attention_bf16_static")
     return o
 
 

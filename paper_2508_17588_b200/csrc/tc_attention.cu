@@ -112,6 +112,9 @@ __device__ __forceinline__ void softmax_tile(uint32_t t_buf, int valid, float c,
   sum_out = (acc0.x + acc0.y) + (acc1.x + acc1.y);
 }
 
+// kPerCtaStatus = false: a CTA that gave up raises the single word *status.
+// kPerCtaStatus = true:  status[0] counts the CTAs that gave up and status[1 + blockIdx.x] records which.
+template <bool kPerCtaStatus>
 __global__ void __launch_bounds__(kAttThreads, 1)
 tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ O, int n_q, int N,
@@ -289,7 +292,10 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   // ---------------------------------------------------------------- teardown
   tc_fence_before();
   __syncthreads();
-  if (threadIdx.x == 0 && *abort_flag) atomicExch(status, 2);
+  if (threadIdx.x == 0 && *abort_flag) {
+    if (kPerCtaStatus) { atomicAdd(status, 1); status[1 + blockIdx.x] = 2; }
+    else atomicExch(status, 2);
+  }
   if (warp == 1) { __syncwarp(); tc_fence_after(); tmem_dealloc(tmem_base, kAttTmemCols); }
 }
 
@@ -318,15 +324,114 @@ int launch_tc_attention(const void* q, const void* k, const void* v, void* o, in
   static std::once_flag attr_once;
   static cudaError_t attr_err = cudaSuccess;
   std::call_once(attr_once, [] {
-    attr_err = cudaFuncSetAttribute(tc_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
+    attr_err = cudaFuncSetAttribute(tc_attention_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)kAttSmem);
   });
   HERO_CUDA_TRY(attr_err);
   const int q_groups = (n_q + kQT * kQTiles - 1) / (kQT * kQTiles);
   const long long grid = (long long)q_groups * heads * B;
-  tc_attention_kernel<<<(unsigned)grid, kAttThreads, kAttSmem, s>>>(tm_q, tm_k, tm_v, (__nv_bfloat16*)o, n_q, N,
-                                                                    heads, d_status);
+  tc_attention_kernel<false><<<(unsigned)grid, kAttThreads, kAttSmem, s>>>(tm_q, tm_k, tm_v, (__nv_bfloat16*)o, n_q,
+                                                                           N, heads, d_status);
   HERO_CUDA_TRY(cudaGetLastError());
   return HERO_OK;
 }
 
 }  // namespace hero
+
+// =============================================================================
+// hero_attention_bf16_static: the same attention, for callers that must not allocate
+// =============================================================================
+// hero_attention_bf16 takes its status word from a cudaMalloc made on first use.  Some
+// callers cannot afford that: a host thread inside a latency-critical serving loop (cudaMalloc
+// and cudaFree synchronise the whole device), a process whose framework has already reserved all
+// device memory for its own pool (the allocation would fail), or code that runs where the CUDA
+// allocator must not be entered at all.  For them the scratch lives in the library image itself:
+// a file-scope __device__ array that every GPU loading the library carries until the process
+// exits (kStaticScratchInts * 4 bytes = 64.25 KiB per GPU).
+//
+// Layout: word 0 counts the CTAs of the latest call that gave up on a bounded wait, word 1 + i
+// records CTA i.  The array is shared by every call and keeps the previous call's contents, so
+// each call clears the words it is going to use on its stream before the kernel runs; two
+// calls that overlap on the GPU (different streams, no dependency) race on it.
+namespace hero {
+namespace {
+
+constexpr int kStaticMaxCtas = 16384;                 // largest grid the static scratch can serve
+constexpr int kStaticScratchInts = 64 + kStaticMaxCtas;
+static __device__ __align__(256) int g_att_static_scratch[kStaticScratchInts];
+
+constexpr int kStaticMaxDevices = 64;
+struct StaticSetup { bool done = false; int* scratch = nullptr; };
+StaticSetup g_static_setup[kStaticMaxDevices];
+std::mutex g_static_mutex;
+
+// Once per device, with that device current: resolve the DEVICE address of the array (in host
+// code the array's name is only a host-side handle, never a pointer a kernel may be given) and
+// raise the kernel's dynamic shared-memory limit.
+int static_setup(int** scratch) {
+  int dev = -1;
+  HERO_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kStaticMaxDevices) return HERO_ERR_ARG;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  StaticSetup& st = g_static_setup[dev];
+  if (!st.done) {
+    int* p = nullptr;
+    HERO_CUDA_TRY(cudaGetSymbolAddress((void**)&p, g_att_static_scratch));
+    HERO_CUDA_TRY(cudaFuncSetAttribute(tc_attention_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)kAttSmem));
+    st.scratch = p;
+    st.done = true;
+  }
+  *scratch = st.scratch;
+  return HERO_OK;
+}
+
+}  // namespace
+}  // namespace hero
+
+extern "C" int hero_attention_bf16_static(const void* d_q, const void* d_k, const void* d_v, void* d_o, int B,
+                                          int n_q, int N, int heads, void* stream, int* h_gave_up) {
+  using namespace hero;
+  if (h_gave_up) *h_gave_up = 0;
+  if (B < 0 || n_q < 0 || N <= 0 || heads <= 0) return HERO_ERR_ARG;
+  if (B == 0 || n_q == 0) return HERO_OK;
+  if (!d_q || !d_k || !d_v || !d_o) return HERO_ERR_ARG;
+  if (!aligned16(d_q) || !aligned16(d_k) || !aligned16(d_v) || !aligned16(d_o)) return HERO_ERR_ALIGN;
+  const long long q_groups = ((long long)n_q + kQT * kQTiles - 1) / (kQT * kQTiles);
+  const long long grid = q_groups * heads * B;
+  if (grid > kStaticMaxCtas) {
+    set_cuda_error(cudaErrorInvalidConfiguration,
+                   "hero_attention_bf16_static: ceil(n_q/256)*heads*B exceeds the 16384 CTAs its static scratch "
+                   "serves; split the call or use hero_attention_bf16");
+    return HERO_ERR_CAP;
+  }
+  cudaStream_t s = (cudaStream_t)stream;
+  int* scratch = nullptr;
+  HERO_TRY(static_setup(&scratch));
+  const uint64_t D = (uint64_t)heads * kHD;
+  CUtensorMap tm_q, tm_k, tm_v;
+  {
+    const uint64_t dims[2] = {D, (uint64_t)B * n_q};
+    const uint64_t str[1] = {D * 2};
+    const uint32_t box[2] = {(uint32_t)kHD, (uint32_t)kQT};
+    HERO_TRY(make_tmap_bf16(&tm_q, d_q, 2, dims, str, box));
+  }
+  {
+    const uint64_t dims[3] = {D, (uint64_t)N, (uint64_t)B};
+    const uint64_t str[2] = {D * 2, (uint64_t)N * D * 2};
+    const uint32_t box[3] = {(uint32_t)kHD, (uint32_t)kKT, 1};
+    HERO_TRY(make_tmap_bf16(&tm_k, d_k, 3, dims, str, box));
+    HERO_TRY(make_tmap_bf16(&tm_v, d_v, 3, dims, str, box));
+  }
+  // the array still holds the previous call's records: clear the words this grid will use
+  HERO_CUDA_TRY(cudaMemsetAsync(scratch, 0, (size_t)(1 + grid) * sizeof(int), s));
+  tc_attention_kernel<true><<<(unsigned)grid, kAttThreads, kAttSmem, s>>>(tm_q, tm_k, tm_v, (__nv_bfloat16*)d_o, n_q,
+                                                                          N, heads, scratch);
+  HERO_CUDA_TRY(cudaGetLastError());
+  if (h_gave_up) {
+    HERO_CUDA_TRY(cudaMemcpyAsync(h_gave_up, scratch, sizeof(int), cudaMemcpyDeviceToHost, s));
+    HERO_CUDA_TRY(cudaStreamSynchronize(s));
+    if (*h_gave_up != 0) return HERO_ERR_TIMEOUT;
+  }
+  return HERO_OK;
+}
