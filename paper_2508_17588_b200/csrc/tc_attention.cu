@@ -3,23 +3,42 @@
 // no score matrix ever leaves the SM.
 //
 // One CTA = 256 query rows (two tiles of 128) of one (batch, head); it streams all N cached
-// keys in tiles of 128 through a 4-stage TMA ring shared by both query tiles.
-//   warp 0      TMA: both Q tiles once, then K/V tiles (128-byte swizzle)
-//   warp 1      tcgen05.mma issuer: S = Q K^T (M128 N128 K64) into TMEM, then P V (M128 N64 K128)
-//               with P read from TMEM and V as an N-contiguous shared-memory operand
-//   warps 2..5  softmax group of query tile 0, warps 6..9 of query tile 1: one thread per
-//               query row; running max / sum in registers, P written back over S in TMEM as
-//               bf16, the running output rescaled and accumulated in registers
-// TMEM holds four 128-column buffers, (query tile) x (key tile parity).  A buffer first receives
-// S; the softmax overwrites columns [0,64) with P; the P V product lands in columns [64,128).
-// Two softmax groups keep every SM sub-partition busy while the other group waits on the
-// tensor core.
+// keys in tiles of 96 through a 6-stage TMA ring shared by both query tiles.
+//   warp 0        TMA: both Q tiles once, then K/V tiles (128-byte swizzle)
+//   warp 1, 2     tcgen05.mma issuers, one thread per query tile: S = Q K^T (M128 N96 K64) into
+//                 TMEM, then O += P V (M128 N64 K96) with P read from TMEM and V as an
+//                 N-contiguous shared-memory operand.  Each tile has its own issuer so that
+//                 neither tile's hand-shakes can hold up the other's.
+//   warps 4..7    softmax group of query tile 0, warps 8..11 of query tile 1: one thread per
+//                 query row, which holds the row's 96 scores of a key tile in registers (one TMEM
+//                 read burst per tile); running max / sum in registers, P written back over S
+//                 in TMEM as bf16
+// TMEM (512 columns): per query tile two S buffers of 96 columns (key tile parity) and one
+// 64-column output accumulator; P (48 columns of bf16 pairs) overwrites the head of its S buffer.
+//
+// Nothing on the per-tile path waits for the tensor core in steady state:
+//   * S of tile j+2 is issued right after P V of tile j, into the buffer whose P that product
+//     reads (MMAs of one issuer execute in issue order), i.e. a whole softmax iteration before
+//     it is needed;
+//   * the output accumulates in TMEM across key tiles, and the running maximum that scales P
+//     is only moved when a tile's maximum exceeds it by more than 2^8 (P stays far inside the
+//     bf16 / fp32 range); only then is the accumulator multiplied down, after the previous
+//     P V has completed.  The final division by the row sum makes the result independent of
+//     which maximum was used.
+//
+// The exponential unit, not the tensor core, bounds this kernel at head_dim 64 (one ex2 per 256
+// tensor flops): kPolyOf8 of every 8 score pairs take 2^x from a degree-3 polynomial on the FMA
+// pipe instead (Cody-Waite split x = n + f, |f| <= 1/2, exponent bits added as an integer).
 #include <cuda.h>
 
 #include <mutex>
 
 #include "hero_internal.h"
 #include "tc_common.cuh"
+
+#ifndef HERO_ATT_POLY_OF_8
+#define HERO_ATT_POLY_OF_8 2
+#endif
 
 namespace hero {
 
@@ -29,17 +48,29 @@ int make_tmap_bf16(CUtensorMap* m, const void* base, int rank, const uint64_t* d
 namespace {
 using namespace tc;
 
-constexpr int kQT = 128, kQTiles = 2, kKT = 128, kHD = 64, kKvStages = 4;
+constexpr int kQT = 128, kQTiles = 2, kKT = 96, kHD = 64, kKvStages = 6;
 constexpr int kQBytes = kQT * kHD * 2;       // 16 KB per query tile
-constexpr int kKBytes = kKT * kHD * 2;       // 16 KB
+constexpr int kKBytes = kKT * kHD * 2;       // 12 KB (a multiple of the 1024-byte swizzle atom)
 constexpr int kKvStageBytes = 2 * kKBytes;   // K tile then V tile
-constexpr int kAttThreads = 64 + 128 * kQTiles;
+constexpr int kFirstSoftmaxWarp = 4;
+constexpr int kAttThreads = 32 * (kFirstSoftmaxWarp + 4 * kQTiles);   // 12 warps
 constexpr size_t kAttSmem = 1024 + kQTiles * kQBytes + (size_t)kKvStages * kKvStageBytes + 512;
-constexpr uint32_t kBufCols = 128, kColPV = 64, kAttTmemCols = 512;
+constexpr uint32_t kTileCols = 256, kColO = 2 * kKT, kAttTmemCols = 512;   // per tile: S0 | S1 | O
+constexpr int kPolyOf8 = HERO_ATT_POLY_OF_8;   // score pairs per 8 whose 2^x comes from the polynomial
+constexpr float kRescaleLog2 = 8.0f;           // the scaling maximum moves only when exceeded by 2^8
+static_assert(2 * kKT + kHD <= (int)kTileCols && kQTiles * kTileCols <= kAttTmemCols, "TMEM layout");
+static_assert(kKBytes % 1024 == 0 && kKT % 16 == 0, "tile shape");
 
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// The same instruction, pinned: the compiler keeps volatile statements in program order, which is how
+// the fused pass below spreads its exponentials evenly through the other arithmetic.
+__device__ __forceinline__ float ex2_pinned(float x) {
+  float y;
+  asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
 __device__ __forceinline__ float max3(float a, float b, float c) {
@@ -49,67 +80,126 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 }
 __device__ __forceinline__ float2 f2(uint32_t a, uint32_t b) { return make_float2(__uint_as_float(a), __uint_as_float(b)); }
 
-// One key tile of one query row: S (128 fp32 in TMEM) -> running max, P (bf16 pairs written over
-// the first 64 columns), row sum of P.  `valid` < 128 only in the ragged last tile.
+// 2^x for a pair, x <= 8, on the FMA and integer pipes.  x is clamped at -126 so that the
+// exponent arithmetic stays inside the normal range; t = x + 1.5*2^23 holds round(x) in its low
+// mantissa bits, f = x - round(x) lies in [-1/2, 1/2], the cubic (minimax in relative error,
+// 7.5e-5, far below the bf16 rounding of P) gives 2^f, and round(x) is added to the exponent field.
+__device__ __forceinline__ float2 exp2_poly(float2 x) {
+  const float kMagic = 12582912.0f;
+  x.x = fmaxf(x.x, -126.0f);
+  x.y = fmaxf(x.y, -126.0f);
+  const float2 t = __fadd2_rn(x, make_float2(kMagic, kMagic));
+  const float2 n = __fadd2_rn(t, make_float2(-kMagic, -kMagic));
+  const float2 f = __ffma2_rn(n, make_float2(-1.0f, -1.0f), x);
+  float2 p = __ffma2_rn(f, make_float2(0.0551716648042202f, 0.0551716648042202f),
+                        make_float2(0.2426111251115799f, 0.2426111251115799f));
+  p = __ffma2_rn(p, f, make_float2(0.6932609677314758f, 0.6932609677314758f));
+  p = __ffma2_rn(p, f, make_float2(0.9999280571937561f, 0.9999280571937561f));
+  return make_float2(__uint_as_float(__float_as_uint(p.x) + (__float_as_uint(t.x) << 23)),
+                     __uint_as_float(__float_as_uint(p.y) + (__float_as_uint(t.y) << 23)));
+}
+
+// One key tile of one query row.  The kKT scores of the row are read from TMEM in one burst
+// (a single wait for the whole row instead of one per chunk), reduced to their maximum, turned
+// into p = 2^(s*c - m*c) and written back as bf16 pairs over columns [0, kKT/2) of the same
+// buffer.  m_used is the maximum the row's P and accumulator are scaled by: it only moves when
+// this tile exceeds it by more than 2^kRescaleLog2 (always at the first tile), and alpha is then
+// the factor that the sum and the accumulator take.  Returns the row sum of p.
 template <bool MASKED>
-__device__ __forceinline__ void softmax_tile(uint32_t t_buf, int valid, float c, float& m_run, float& alpha_out,
-                                             float& sum_out) {
-  // pass 1: row maximum (two independent chains, three-input max)
-  float mx0 = -INFINITY, mx1 = -INFINITY;
-#pragma unroll 1
-  for (int ch = 0; ch < kKT / 32; ++ch) {
-    uint32_t r[32];
-    tmem_ld32(t_buf + ch * 32, r);
-    tmem_ld_wait();
-    if (MASKED) {
+__device__ __forceinline__ float softmax_tile(uint32_t t_buf, int valid, float c, float& m_used, float& alpha,
+                                              bool& grow) {
+  uint32_t s[kKT];
 #pragma unroll
-      for (int i = 0; i < 32; ++i)
-        if (ch * 32 + i >= valid) r[i] = 0xFF800000u;   // -inf
-    }
+  for (int ch = 0; ch < kKT / 32; ++ch) tmem_ld32(t_buf + ch * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[ch * 32]));
+  tmem_ld_wait();
+  if (MASKED) {
 #pragma unroll
-    for (int i = 0; i < 32; i += 4) {
-      mx0 = max3(mx0, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
-      mx1 = max3(mx1, __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
-    }
+    for (int i = 0; i < kKT; ++i)
+      if (i >= valid) s[i] = 0xFF800000u;   // -inf
   }
-  const float m_new = max3(m_run, mx0, mx1);
-  alpha_out = ex2((m_run - m_new) * c);
-  m_run = m_new;
+  float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+  for (int i = 0; i < kKT; i += 8) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) mx[q] = fmaxf(mx[q], fmaxf(__uint_as_float(s[i + 2 * q]), __uint_as_float(s[i + 2 * q + 1])));
+  }
+  const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+  grow = (m_tile - m_used) * c > kRescaleLog2;                 // true at the first tile (m_used = -inf)
+  const float m_new = grow ? m_tile : m_used;
+  alpha = grow ? ex2((m_used - m_new) * c) : 1.0f;             // 0 at the first tile
+  m_used = m_new;
   const float neg_mc = -m_new * c;
   const float2 c2 = make_float2(c, c), nm2 = make_float2(neg_mc, neg_mc);
-  // pass 2: p = 2^(s*c - m*c); bf16 pairs go back into columns [0,64) of the same buffer
-  float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
-#pragma unroll 1
-  for (int half = 0; half < 2; ++half) {
-    uint32_t packed[32];
+  float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
-    for (int sub = 0; sub < 2; ++sub) {
-      uint32_t r[32];
-      tmem_ld32(t_buf + half * 64 + sub * 32, r);
-      tmem_ld_wait();
+  for (int ch = 0; ch < kKT / 32; ++ch) {
+    uint32_t packed[16];
 #pragma unroll
-      for (int i = 0; i < 32; i += 4) {
-        float2 x0 = __ffma2_rn(f2(r[i], r[i + 1]), c2, nm2);
-        float2 x1 = __ffma2_rn(f2(r[i + 2], r[i + 3]), c2, nm2);
-        float2 p0 = make_float2(ex2(x0.x), ex2(x0.y));
-        float2 p1 = make_float2(ex2(x1.x), ex2(x1.y));
-        if (MASKED) {
-          const int col = half * 64 + sub * 32 + i;
-          if (col >= valid) p0.x = 0.f;
-          if (col + 1 >= valid) p0.y = 0.f;
-          if (col + 2 >= valid) p1.x = 0.f;
-          if (col + 3 >= valid) p1.y = 0.f;
-        }
-        acc0 = __fadd2_rn(acc0, p0);
-        acc1 = __fadd2_rn(acc1, p1);
-        const __nv_bfloat162 b0 = __floats2bfloat162_rn(p0.x, p0.y), b1 = __floats2bfloat162_rn(p1.x, p1.y);
-        packed[sub * 16 + i / 2] = *reinterpret_cast<const uint32_t*>(&b0);
-        packed[sub * 16 + i / 2 + 1] = *reinterpret_cast<const uint32_t*>(&b1);
+    for (int i = 0; i < 16; ++i) {       // pair i = columns 2i, 2i+1 of this 32-column chunk
+      const int col = ch * 32 + 2 * i;
+      const float2 x = __ffma2_rn(f2(s[col], s[col + 1]), c2, nm2);
+      float2 p;
+      if (!MASKED && (i & 7) < kPolyOf8) p = exp2_poly(x);
+      else p = make_float2(ex2(x.x), ex2(x.y));
+      if (MASKED) {
+        if (col >= valid) p.x = 0.f;
+        if (col + 1 >= valid) p.y = 0.f;
+      }
+      acc[i & 3] = __fadd2_rn(acc[i & 3], p);
+      const __nv_bfloat162 b = __floats2bfloat162_rn(p.x, p.y);
+      packed[i] = *reinterpret_cast<const uint32_t*>(&b);
+    }
+    tmem_st16(t_buf + ch * 16, packed);
+  }
+  const float2 a01 = __fadd2_rn(acc[0], acc[1]), a23 = __fadd2_rn(acc[2], acc[3]);
+  return (a01.x + a01.y) + (a23.x + a23.y);
+}
+
+// The common case of a key tile, in ONE pass over the row: p = 2^((s - m_used) c) with the maximum
+// the row is already scaled by, the tile's own maximum tracked on the side.  The caller checks the
+// maximum afterwards and falls back to softmax_tile (S is still intact: P is only kept in
+// registers here) in the rare case that it has to move.  Doing without the separate maximum pass
+// matters because that pass issues nothing to the exponential unit: two warps of an SM
+// sub-partition then tend to run their exponential phases at the same time and their other
+// phases at the same time, and the unit that bounds the kernel idles in between.  Here every
+// stretch of the instruction stream has the same mix: the exponentials are issued in a fixed
+// order, two pairs behind the multiply that feeds them and three pairs ahead of the code that
+// consumes them, with the scores read 32 columns at a time one chunk ahead.
+__device__ __forceinline__ void fused_tile(uint32_t t_buf, float c, float neg_mc, uint32_t (&packed)[kKT / 2],
+                                           float& sum, float& m_tile) {
+  const float2 c2 = make_float2(c, c), nm2 = make_float2(neg_mc, neg_mc);
+  float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+  float mx[2] = {-INFINITY, -INFINITY};
+  uint32_t ra[32], rb[32];
+  tmem_ld32(t_buf, ra);
+#pragma unroll
+  for (int ch = 0; ch < kKT / 32; ++ch) {
+    uint32_t(&cur)[32] = (ch & 1) ? rb : ra;
+    uint32_t(&nxt)[32] = (ch & 1) ? ra : rb;
+    tmem_ld_wait();
+    if (ch + 1 < kKT / 32) tmem_ld32(t_buf + (ch + 1) * 32, nxt);
+    float2 x[16], p[16];
+    x[0] = __ffma2_rn(f2(cur[0], cur[1]), c2, nm2);
+    x[1] = __ffma2_rn(f2(cur[2], cur[3]), c2, nm2);
+#pragma unroll
+    for (int i = 0; i < 16 + 3; ++i) {
+      if (i + 2 < 16) x[i + 2] = __ffma2_rn(f2(cur[2 * i + 4], cur[2 * i + 5]), c2, nm2);
+      if (i < 16) {
+        if ((i & 7) < kPolyOf8) p[i] = exp2_poly(x[i]);
+        else { p[i].x = ex2_pinned(x[i].x); p[i].y = ex2_pinned(x[i].y); }
+      }
+      if (i >= 3) {
+        const int k = i - 3;
+        acc[k & 3] = __fadd2_rn(acc[k & 3], p[k]);
+        const __nv_bfloat162 b = __floats2bfloat162_rn(p[k].x, p[k].y);
+        packed[ch * 16 + k] = *reinterpret_cast<const uint32_t*>(&b);
+        mx[k & 1] = max3(mx[k & 1], __uint_as_float(cur[2 * k]), __uint_as_float(cur[2 * k + 1]));
       }
     }
-    tmem_st32(t_buf + half * 32, packed);
   }
-  sum_out = (acc0.x + acc0.y) + (acc1.x + acc1.y);
+  const float2 a01 = __fadd2_rn(acc[0], acc[1]), a23 = __fadd2_rn(acc[2], acc[3]);
+  sum = (a01.x + a01.y) + (a23.x + a23.y);
+  m_tile = fmaxf(mx[0], mx[1]);
 }
 
 // kPerCtaStatus = false: a CTA that gave up raises the single word *status.
@@ -125,13 +215,12 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   uint8_t* s_kv = smem + kQTiles * kQBytes;
   uint64_t* bars = reinterpret_cast<uint64_t*>(s_kv + (size_t)kKvStages * kKvStageBytes);
   uint64_t* q_full = bars;
-  uint64_t* kv_full = bars + 1;                    // [kKvStages]
-  uint64_t* kv_empty = kv_full + kKvStages;        // [kKvStages]
-  uint64_t* s_full = kv_empty + kKvStages;         // [qt][parity]  MMA -> softmax: S is ready
-  uint64_t* p_full = s_full + 4;                   // [qt][parity]  softmax -> MMA: P is in TMEM
-  uint64_t* pv_full = p_full + 4;                  // [qt][parity]  MMA -> softmax: P V is ready
-  uint64_t* o_done = pv_full + 4;                  // [qt][parity]  softmax -> MMA: buffer may be reused
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_done + 4);
+  uint64_t* kv_full = bars + 1;                    // [kKvStages]           TMA -> both issuers
+  uint64_t* kv_empty = kv_full + kKvStages;        // [kKvStages], count 2  both issuers -> TMA
+  uint64_t* s_full = kv_empty + kKvStages;         // [qt][parity]  issuer -> softmax: S is ready
+  uint64_t* p_full = s_full + 4;                   // [qt][parity]  softmax -> issuer: P is in TMEM
+  uint64_t* pv_full = p_full + 4;                  // [qt]          issuer -> softmax: P V of tile j done (phase j)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(pv_full + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -143,10 +232,9 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
-    for (int i = 0; i < kKvStages; ++i) { mbar_init(&kv_full[i], 1); mbar_init(&kv_empty[i], 1); }
-    for (int i = 0; i < 4; ++i) {
-      mbar_init(&s_full[i], 1); mbar_init(&p_full[i], 4); mbar_init(&pv_full[i], 1); mbar_init(&o_done[i], 4);
-    }
+    for (int i = 0; i < kKvStages; ++i) { mbar_init(&kv_full[i], 1); mbar_init(&kv_empty[i], kQTiles); }
+    for (int i = 0; i < 4; ++i) { mbar_init(&s_full[i], 1); mbar_init(&p_full[i], 4); }
+    for (int i = 0; i < kQTiles; ++i) mbar_init(&pv_full[i], 1);
     *abort_flag = 0;
     mbar_fence_init();
   }
@@ -177,113 +265,133 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (++stage == kKvStages) { stage = 0; phase ^= 1; }
       }
     }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
+  } else if (warp == 1 || warp == 2) {
+    // ------------------------------------------------------------ MMA issuer of query tile t
     if (lane == 0) {
+      const int t = warp - 1;
       constexpr uint32_t idesc_s = idesc_bf16(kQT, kKT, 0);    // S = Q K^T : both operands K-contiguous
-      constexpr uint32_t idesc_pv = idesc_bf16(kQT, kHD, 1);   // O = P V   : V is N(head_dim)-contiguous
-      auto issue_s = [&](int t, int j) {
+      constexpr uint32_t idesc_pv = idesc_bf16(kQT, kHD, 1);   // O += P V  : V is N(head_dim)-contiguous
+      const uint64_t dq = smem_desc_sw128(smem_u32(s_q + t * kQBytes), 1024);
+      const uint32_t t_tile = tmem_base + (uint32_t)t * kTileCols;
+      auto issue_s = [&](int j) {
         const int st = j % kKvStages;
-        const uint64_t dq = smem_desc_sw128(smem_u32(s_q + t * kQBytes), 1024);
         const uint64_t dk = smem_desc_sw128(smem_u32(s_kv + (size_t)st * kKvStageBytes), 1024);
-        const uint32_t d = tmem_base + (uint32_t)(t * 2 + (j & 1)) * kBufCols;
+        const uint32_t d = t_tile + (uint32_t)(j & 1) * kKT;
 #pragma unroll
         for (int k = 0; k < kHD / 16; ++k) mma_ss(d, dq + 2 * k, dk + 2 * k, idesc_s, k != 0);
         mma_commit(&s_full[t * 2 + (j & 1)]);
       };
       bool ok = mbar_wait(q_full, 0, abort_flag);
-      if (ok) ok = mbar_wait(&kv_full[0], 0, abort_flag);
-      if (ok) { tc_fence_after(); issue_s(0, 0); issue_s(1, 0); }
+      for (int j = 0; j < 2 && j < n_kv && ok; ++j) {           // two score tiles ahead of the softmax
+        if ((ok = mbar_wait(&kv_full[j], 0, abort_flag))) { tc_fence_after(); issue_s(j); }
+      }
       for (int j = 0; j < n_kv && ok; ++j) {
-        if (j + 1 < n_kv) {
-          if (!(ok = mbar_wait(&kv_full[(j + 1) % kKvStages], ((j + 1) / kKvStages) & 1, abort_flag))) break;
-          for (int t = 0; t < kQTiles && ok; ++t) {
-            // buffer (t, (j+1)&1) last held tile j-1: its P V must have been read out
-            if (j >= 1) ok = mbar_wait(&o_done[t * 2 + ((j + 1) & 1)], ((j - 1) >> 1) & 1, abort_flag);
-            if (ok) { tc_fence_after(); issue_s(t, j + 1); }
-          }
-          if (!ok) break;
-        }
         const int st = j % kKvStages;
         // V tile: rows = keys (128 bytes each), 8-key groups 1024 bytes apart; 16 keys per MMA = 2048 bytes
         const uint64_t dv = smem_desc_sw128(smem_u32(s_kv + (size_t)st * kKvStageBytes + kKBytes), 1024);
-        for (int t = 0; t < kQTiles && ok; ++t) {
-          const int bi = t * 2 + (j & 1);
-          if (!(ok = mbar_wait(&p_full[bi], (j >> 1) & 1, abort_flag))) break;
-          tc_fence_after();
-          const uint32_t buf = tmem_base + (uint32_t)bi * kBufCols;
+        if (!(ok = mbar_wait(&p_full[t * 2 + (j & 1)], (j >> 1) & 1, abort_flag))) break;
+        tc_fence_after();
+        const uint32_t buf = t_tile + (uint32_t)(j & 1) * kKT;
 #pragma unroll
-          for (int k = 0; k < kKT / 16; ++k) mma_ts(buf + kColPV, buf + 8 * k, dv + 128 * k, idesc_pv, k != 0);
-          mma_commit(&pv_full[bi]);
+        for (int k = 0; k < kKT / 16; ++k) mma_ts(t_tile + kColO, buf + 8 * k, dv + 128 * k, idesc_pv, (j | k) != 0);
+        mma_commit(&pv_full[t]);
+        mma_commit(&kv_empty[st]);               // second arrival comes from the other tile's issuer
+        if (j + 2 < n_kv) {
+          // S of tile j+2 overwrites the buffer whose P the product above reads: safe because the
+          // tensor core executes this thread's MMAs in issue order
+          if (!(ok = mbar_wait(&kv_full[(j + 2) % kKvStages], ((j + 2) / kKvStages) & 1, abort_flag))) break;
+          tc_fence_after();
+          issue_s(j + 2);
         }
-        if (ok) mma_commit(&kv_empty[st]);
       }
     }
-  } else {
-    // ------------------------------------------------------------ softmax + output accumulation
-    const int t = (warp - 2) >> 2;                     // query tile of this softmax group
+  } else if (warp >= kFirstSoftmaxWarp) {
+    // ------------------------------------------------------------ softmax
+    const int t = (warp - kFirstSoftmaxWarp) >> 2;     // query tile of this softmax group
     const int quad = warp & 3;                         // TMEM lane quadrant this warp may touch
-    const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(t * 2) * kBufCols;
+    const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)t * kTileCols;
     const float c = 0.125f * 1.4426950408889634f;      // 1/sqrt(64) * log2(e)
-    float m_run = -INFINITY, l_run = 0.f, alpha_pend = 0.f;
-    float2 o[kHD / 2];
-#pragma unroll
-    for (int i = 0; i < kHD / 2; ++i) o[i] = make_float2(0.f, 0.f);
-    auto fold_pv = [&](int j) -> bool {                // O = O * alpha + (P V)_j, then release the buffer
-      bool good = mbar_wait(&pv_full[t * 2 + (j & 1)], (j >> 1) & 1, abort_flag);
-      good = __all_sync(0xFFFFFFFFu, good);
-      if (!good) return false;
-      tc_fence_after();
-      const uint32_t t_pv = lane_base + (uint32_t)(j & 1) * kBufCols + kColPV;
-      uint32_t r0[32], r1[32];
-      tmem_ld32(t_pv, r0);
-      tmem_ld32(t_pv + 32, r1);
-      tmem_ld_wait();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&o_done[t * 2 + (j & 1)]);
-      const float2 a2 = make_float2(alpha_pend, alpha_pend);
-#pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        o[i] = __ffma2_rn(o[i], a2, f2(r0[2 * i], r0[2 * i + 1]));
-        o[16 + i] = __ffma2_rn(o[16 + i], a2, f2(r1[2 * i], r1[2 * i + 1]));
-      }
-      return true;
-    };
+    float m_used = -INFINITY, l_run = 0.f;
     bool ok = true;
     for (int j = 0; j < n_kv; ++j) {
       ok = mbar_wait(&s_full[t * 2 + (j & 1)], (j >> 1) & 1, abort_flag);
       ok = __all_sync(0xFFFFFFFFu, ok);
       if (!ok) break;
       tc_fence_after();
-      const uint32_t t_buf = lane_base + (uint32_t)(j & 1) * kBufCols;
+      const uint32_t t_buf = lane_base + (uint32_t)(j & 1) * kKT;
       const int valid = N - j * kKT;                   // keys of this tile that exist (>= 1)
-      float alpha, sum;
-      if (valid >= kKT) softmax_tile<false>(t_buf, valid, c, m_run, alpha, sum);
-      else softmax_tile<true>(t_buf, valid, c, m_run, alpha, sum);
+      const bool ragged = valid < kKT;
+      float alpha = 1.0f, sum;
+      bool grow = true;                                // first and ragged tiles take the two-pass path
+      uint32_t packed[kKT / 2];
+      if (j > 0 && !ragged) {
+        float m_tile;
+        fused_tile(t_buf, c, -m_used * c, packed, sum, m_tile);
+        grow = __any_sync(0xFFFFFFFFu, (m_tile - m_used) * c > kRescaleLog2);
+      }
+      if (grow) {                                      // warp-uniform
+        bool moved;
+        sum = ragged ? softmax_tile<true>(t_buf, valid, c, m_used, alpha, moved)
+                     : softmax_tile<false>(t_buf, valid, c, m_used, alpha, moved);
+      } else {
+#pragma unroll
+        for (int ch = 0; ch < kKT / 32; ++ch)
+          tmem_st16(t_buf + ch * 16, *reinterpret_cast<uint32_t(*)[16]>(&packed[ch * 16]));
+      }
+      l_run = fmaf(l_run, alpha, sum);
+      if (j > 0) {
+        // P V of the previous tile was issued a whole iteration ago; observe its completion (every
+        // phase of the barrier is consumed) and, in the rare case the maximum moved, scale the
+        // accumulator down before this tile's product is added to it
+        ok = mbar_wait(&pv_full[t], (j - 1) & 1, abort_flag);
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) break;
+        if (grow) {                                    // warp-uniform; alpha is 1 for rows that did not move
+          tc_fence_after();
+          const float2 a2 = make_float2(alpha, alpha);
+#pragma unroll
+          for (int ch = 0; ch < kHD / 16; ++ch) {
+            uint32_t r[16];
+            tmem_ld16(lane_base + kColO + ch * 16, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 16; i += 2) {
+              const float2 v = __fmul2_rn(f2(r[i], r[i + 1]), a2);
+              r[i] = __float_as_uint(v.x); r[i + 1] = __float_as_uint(v.y);
+            }
+            tmem_st16(lane_base + kColO + ch * 16, r);
+          }
+        }
+      }
       tmem_st_wait();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&p_full[t * 2 + (j & 1)]);
-      // fold in the previous tile's P V while the tensor core works on this one
-      if (j > 0 && !(ok = fold_pv(j - 1))) break;
-      l_run = fmaf(l_run, alpha, sum);
-      alpha_pend = alpha;
     }
-    if (ok && fold_pv(n_kv - 1)) {
+    if (ok) {
+      ok = mbar_wait(&pv_full[t], (n_kv - 1) & 1, abort_flag);
+      ok = __all_sync(0xFFFFFFFFu, ok);
+    }
+    if (ok) {
+      tc_fence_after();
       const int qi = (qg * kQTiles + t) * kQT + quad * 32 + lane;
-      if (qi < n_q) {
-        const float inv = 1.0f / l_run;
-        __nv_bfloat16* dst = O + ((long long)b * n_q + qi) * ((long long)heads * kHD) + h * kHD;
+      const float inv = 1.0f / l_run;
+      __nv_bfloat16* dst = O + ((long long)b * n_q + qi) * ((long long)heads * kHD) + h * kHD;
 #pragma unroll
-        for (int v = 0; v < kHD / 8; ++v) {
-          uint32_t w[4];
+      for (int ch = 0; ch < kHD / 16; ++ch) {
+        uint32_t r[16];
+        tmem_ld16(lane_base + kColO + ch * 16, r);     // warp-collective: every lane loads
+        tmem_ld_wait();
+        if (qi < n_q) {
+          uint32_t w[8];
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const __nv_bfloat162 pk = __floats2bfloat162_rn(o[v * 4 + q].x * inv, o[v * 4 + q].y * inv);
+          for (int q = 0; q < 8; ++q) {
+            const __nv_bfloat162 pk = __floats2bfloat162_rn(__uint_as_float(r[2 * q]) * inv,
+                                                            __uint_as_float(r[2 * q + 1]) * inv);
             w[q] = *reinterpret_cast<const uint32_t*>(&pk);
           }
-          *reinterpret_cast<uint4*>(dst + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(dst + ch * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(dst + ch * 16 + 8) = make_uint4(w[4], w[5], w[6], w[7]);
         }
       }
     }
