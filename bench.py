@@ -357,10 +357,12 @@ def run_hero(args, cfg, rank, world, local_rank):
 
 # --------------------------------------------------------------------------- isolated kernels
 def _time_flushed(fn, iters, warmup, flush):
-    """Median device time (ms) of fn() with L2 flushed (a write larger than L2) before each call."""
+    """Median device time (ms) of fn() with L2 flushed before each call: a write larger than L2, then a
+    read of the same buffer so that what L2 is left holding is clean (evicting it costs no write-back)."""
     ts = []
     for i in range(warmup + iters):
         flush.zero_()
+        flush.max()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         fn()
@@ -483,7 +485,7 @@ def run_kernels(args):
             tensor(f"refresh_block_{num}/{den}", ms, fl["gemm"] + fl["attention"], n_sel=state["n"])
             hero.close()
     print(json.dumps({"workload": "kernels", "small": bool(args.small), "iters": iters, "timing":
-                      "CUDA events, median, L2 flushed by a 256 MiB write before every call",
+                      "CUDA events, median, L2 flushed by a 256 MiB write + read before every call",
                       "peaks": peaks, "kernels": out}))
 
 

@@ -202,8 +202,10 @@ __global__ void __launch_bounds__(kStreamThreads) residual2_kernel(T* __restrict
 }
 
 // ------------------------------------------------------------------ gather / scatter of rows
-// One warp moves one row in 16-byte packets; GATHER reads row idx[i] and writes row i,
-// SCATTER the reverse.  Rows not listed are never touched.
+// One warp moves one row in 16-byte packets, four packets per lane in flight at a time (2 KB per
+// warp, 16 KB per CTA); GATHER reads row idx[i] and writes row i, SCATTER the reverse.  Rows not
+// listed are never touched.
+constexpr int kMoveUnroll = 4;
 template <bool GATHER>
 __global__ void __launch_bounds__(256) move_rows_kernel(const uint4* __restrict__ src, const int* __restrict__ idx,
                                                         uint4* __restrict__ dst, int B, int N, int n_sel,
@@ -214,10 +216,18 @@ __global__ void __launch_bounds__(256) move_rows_kernel(const uint4* __restrict_
   const long long total = (long long)B * n_sel;
   for (long long m = warp_global; m < total; m += n_warps) {
     const int b = (int)(m / n_sel), i = (int)(m - (long long)b * n_sel);
-    const long long far = ((long long)b * N + idx[i]) * row_vec, near = m * row_vec;
+    const long long far = ((long long)b * N + __ldg(idx + i)) * row_vec, near = m * row_vec;
     const uint4* s = src + (GATHER ? far : near);
     uint4* d = dst + (GATHER ? near : far);
-    for (int c = lane; c < row_vec; c += 32) __stcs(d + c, __ldcs(s + c));
+    for (int c0 = lane; c0 < row_vec; c0 += 32 * kMoveUnroll) {
+      uint4 v[kMoveUnroll];
+#pragma unroll
+      for (int u = 0; u < kMoveUnroll; ++u)
+        if (c0 + 32 * u < row_vec) v[u] = __ldcs(s + c0 + 32 * u);
+#pragma unroll
+      for (int u = 0; u < kMoveUnroll; ++u)
+        if (c0 + 32 * u < row_vec) __stcs(d + c0 + 32 * u, v[u]);
+    }
   }
 }
 
@@ -334,6 +344,84 @@ gather_ln_modulate_kernel(const T* __restrict__ x, const T* __restrict__ add, co
   }
 }
 
+// bf16 rows of 256 * VPL elements: one WARP per refreshed row, the row held in registers (VPL
+// 16-byte packets per lane), statistics by warp shuffles alone - no shared memory, no block barrier,
+// 8 independent rows in flight per CTA.
+template <int VPL>
+__global__ void __launch_bounds__(256, (VPL > 12) ? 1 : 2)
+gather_ln_modulate_warp_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ add,
+                               const int* __restrict__ idx, const float* __restrict__ shift,
+                               const float* __restrict__ scale, int mod_ld, __nv_bfloat16* __restrict__ a, int N,
+                               int n_sel, long long rows, float eps) {
+  using V = Vec<__nv_bfloat16>;
+  constexpr int D = VPL * 256;
+  const int lane = threadIdx.x & 31;
+  const long long m = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (m >= rows) return;
+  const int b = (int)(m / n_sel), i = (int)(m - (long long)b * n_sel);
+  const long long row = (long long)b * N + (idx ? __ldg(idx + i) : i);
+  const V* xr = reinterpret_cast<const V*>(x + row * D);
+  V raw[VPL];
+#pragma unroll
+  for (int c = 0; c < VPL; ++c) raw[c].raw = __ldcs(&xr[c * 32 + lane].raw);
+  float f[VPL][8];
+#pragma unroll
+  for (int c = 0; c < VPL; ++c) raw[c].unpack(f[c]);
+  if (add) {
+    const V* ar = reinterpret_cast<const V*>(add + row * D);
+#pragma unroll
+    for (int c = 0; c < VPL; ++c) raw[c].raw = __ldcs(&ar[c * 32 + lane].raw);
+#pragma unroll
+    for (int c = 0; c < VPL; ++c) {
+      float g[8];
+      raw[c].unpack(g);
+#pragma unroll
+      for (int q = 0; q < 8; ++q) f[c][q] += g[q];
+    }
+  }
+  float sum = 0.f;
+#pragma unroll
+  for (int c = 0; c < VPL; ++c)
+#pragma unroll
+    for (int q = 0; q < 8; ++q) sum += f[c][q];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+  const float mean = sum / (float)D;
+  float sq = 0.f;
+#pragma unroll
+  for (int c = 0; c < VPL; ++c)
+#pragma unroll
+    for (int q = 0; q < 8; ++q) { const float d = f[c][q] - mean; sq = fmaf(d, d, sq); }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xFFFFFFFFu, sq, o);
+  const float rstd = 1.0f / sqrtf(sq / (float)D + eps);
+  const float4* sh = reinterpret_cast<const float4*>(shift + (long long)b * mod_ld);
+  const float4* sc = reinterpret_cast<const float4*>(scale + (long long)b * mod_ld);
+  V* out = reinterpret_cast<V*>(a + m * D);
+#pragma unroll
+  for (int c = 0; c < VPL; ++c) {
+    const int v = c * 32 + lane;       // packet index: columns [8v, 8v + 8)
+    const float4 s0 = __ldg(sc + 2 * v), s1 = __ldg(sc + 2 * v + 1), h0 = __ldg(sh + 2 * v), h1 = __ldg(sh + 2 * v + 1);
+    const float scl[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+    const float sft[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
+    float r[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) r[q] = fmaf((f[c][q] - mean) * rstd, 1.0f + scl[q], sft[q]);
+    V o; o.pack(r);
+    out[v] = o;
+  }
+}
+
+template <int VPL>
+int gather_ln_warp(const void* x, const void* add, const int* idx, const float* shift, const float* scale, int mod_ld,
+                   void* a, int N, int n_sel, long long rows, float eps, cudaStream_t s) {
+  using T = __nv_bfloat16;
+  gather_ln_modulate_warp_kernel<VPL><<<(unsigned)((rows + 7) / 8), 256, 0, s>>>(
+      (const T*)x, (const T*)add, idx, shift, scale, mod_ld, (T*)a, N, n_sel, rows, eps);
+  HERO_CUDA_TRY(cudaGetLastError());
+  return HERO_OK;
+}
+
 template <typename T>
 int extrapolate_t(const void* p, const void* l, void* o, long long n, float c, cudaStream_t s) {
   extrapolate_kernel<T><<<stream_grid(n / Vec<T>::N), kStreamThreads, 0, s>>>((const T*)p, (const T*)l, (T*)o, n, c);
@@ -391,7 +479,7 @@ static int move_rows(bool gather, const void* src, const int* idx, void* dst, in
   const long long rows = (long long)B * n_sel;
   if (rows == 0) return HERO_OK;
   long long blocks = (rows + 7) / 8;   // 8 warps per CTA, one row per warp
-  const long long cap = (long long)num_sms() * 8;
+  const long long cap = (long long)num_sms() * 16;
   if (blocks > cap) blocks = cap;
   if (gather)
     move_rows_kernel<true><<<(int)blocks, 256, 0, s>>>((const uint4*)src, idx, (uint4*)dst, B, N, n_sel,
@@ -442,6 +530,12 @@ int launch_gather_ln_modulate(const void* x, const void* add, const int* idx, co
   if (dtype == HERO_DTYPE_BF16) {
     using T = __nv_bfloat16;
     if (D % 8) return HERO_ERR_ALIGN;
+    // the adaLN vectors are read as float4: every block's slice starts 16-byte aligned when mod_ld % 4 == 0
+    const bool vec_ok = mod_ld % 4 == 0 && ((reinterpret_cast<uintptr_t>(shift) | reinterpret_cast<uintptr_t>(scale)) & 15) == 0;
+    if (vec_ok && D == 1024) return gather_ln_warp<4>(x, add, idx, shift, scale, mod_ld, a, N, n_sel, rows, eps, s);
+    if (vec_ok && D == 2048) return gather_ln_warp<8>(x, add, idx, shift, scale, mod_ld, a, N, n_sel, rows, eps, s);
+    if (vec_ok && D == 3072) return gather_ln_warp<12>(x, add, idx, shift, scale, mod_ld, a, N, n_sel, rows, eps, s);
+    if (vec_ok && D == 4096) return gather_ln_warp<16>(x, add, idx, shift, scale, mod_ld, a, N, n_sel, rows, eps, s);
     gather_ln_modulate_kernel<T><<<(unsigned)rows, kLnThreads, smem, s>>>((const T*)x, (const T*)add, idx, shift,
                                                                            scale, mod_ld, (T*)a, N, n_sel, D, eps);
   } else {
