@@ -189,6 +189,26 @@ def run_reference(args, cfg, rank, world):
     print(json.dumps(line))
 
 
+# --------------------------------------------------------------------------- multi-rank plumbing
+def max_over_ranks(value: float, dist, device) -> float:
+    """A timing is the slowest rank's (works on any backend: the tensor lives where `device` says)."""
+    if dist is None:
+        return float(value)
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_throughput(tokens_per_rank_step: int, world: int, ms_per_step: float) -> float:
+    """Independent sequences, one per rank (weak scaling): units of all ranks over the slowest rank's time."""
+    return world * tokens_per_rank_step / (ms_per_step * 1e-3)
+
+
+def rank_seed(base_seed: int, rank: int) -> int:
+    """Each rank draws its own problem."""
+    return base_seed + rank
+
+
 # --------------------------------------------------------------------------- CUDA arm
 def build_device_weights(cfg, device):
     dt = torch.bfloat16 if cfg["dtype"] == "bf16" else torch.float32
@@ -214,7 +234,7 @@ def run_hero(args, cfg, rank, world, local_rank):
         dist.init_process_group("nccl", device_id=device)
     dt = torch.bfloat16 if cfg["dtype"] == "bf16" else torch.float32
     run_cfg = dict(cfg, full_interval=0)         # after the two warm-up full steps every step is cached
-    run_cfg["seed"] = cfg["seed"] + rank         # each rank its own sequence (independent problems)
+    run_cfg["seed"] = rank_seed(cfg["seed"], rank)   # each rank its own sequence (independent problems)
     weights = build_device_weights(run_cfg, device)
     hero = H.Hero(run_cfg, weights)
     B, N, D = cfg["batch"], S.n_rows(cfg), cfg["hidden"]
@@ -259,12 +279,9 @@ def run_hero(args, cfg, rank, world, local_rank):
     launches = hero.hero_launch_count() - launches0
     clocks = sampler.stop()
     hero.hero_check_status()
-    if dist:
-        t = torch.tensor([total_ms], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, dist, device)
     ms_per_step = total_ms / args.steps
-    value = world * tokens / (ms_per_step * 1e-3)
+    value = whole_job_throughput(tokens, world, ms_per_step)
 
     # per-category device time over two more cached steps (events around every launch)
     n_prof = 2
@@ -307,13 +324,10 @@ def run_hero(args, cfg, rank, world, local_rank):
     for _ in range(n_e2e):
         hero.hero_step_host(step, h_x, h_t); step += 1
     e2e_s = (time.perf_counter() - t0) / n_e2e
-    if dist:
-        t = torch.tensor([e2e_s], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_s = max_over_ranks(e2e_s, dist, device)
     xb = h_x.numel() * h_x.element_size()
     tb = h_t.numel() * h_t.element_size()
-    e2e = {"value": world * tokens / e2e_s, "unit": UNIT, "ms_per_step": e2e_s * 1e3,
+    e2e = {"value": whole_job_throughput(tokens, world, e2e_s * 1e3), "unit": UNIT, "ms_per_step": e2e_s * 1e3,
            "h2d_bytes_per_step": xb + tb, "d2h_bytes_per_step": xb}
     hero.hero_check_status()
     mem = hero.hero_device_bytes()
