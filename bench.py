@@ -339,6 +339,30 @@ def run_hero(args, cfg, rank, world, local_rank):
     mem = hero.hero_device_bytes()
     hero.close()
 
+    # the same cached step with the deep stack collapsed to one history pair (a variant: not the headline)
+    collapsed = None
+    if cfg["n_shallow"] < cfg["n_blocks"] and not args.no_collapse:
+        hero = H.Hero(dict(run_cfg, deep_collapse=1), weights)
+        for s_ in range(2):
+            hero.hero_step(s_, x, tembs[s_])
+        st = 2
+        for _ in range(args.warmup):
+            hero.hero_step(st, x, tembs[st % 8]); st += 1
+        n_c = max(2, min(args.steps, 5))
+        torch.cuda.synchronize()
+        e0, e1 = ev(), ev()
+        e0.record()
+        for _ in range(n_c):
+            hero.hero_step(st, x, tembs[st % 8]); st += 1
+        e1.record()
+        torch.cuda.synchronize()
+        hero.hero_check_status()
+        c_ms = max_over_ranks(e0.elapsed_time(e1) / n_c, dist, device)
+        collapsed = {"ms_per_step": c_ms, "value": whole_job_throughput(tokens, world, c_ms), "unit": UNIT,
+                     "device_bytes": hero.hero_device_bytes(),
+                     "note": "deep_collapse=1: Eq. 5 applied once to the fp32 sum of the deep blocks' branch outputs"}
+        hero.close()
+
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         del weights
@@ -366,6 +390,8 @@ def run_hero(args, cfg, rank, world, local_rank):
                            "schedule": "%d full + %d cached of %d steps" % (n_full, cfg["steps"] - n_full, cfg["steps"]),
                            "device_bytes": mem, "parallelism": "replicas" if world > 1 else "single"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "breakdown_ms": breakdown}
+        if collapsed:
+            line["deep_collapse_variant"] = collapsed
         if roofline:
             line["roofline"] = roofline
         if cpu_baseline:
@@ -520,6 +546,7 @@ def main():
                                                "attention,gemm,block")
     ap.add_argument("--small", action="store_true", help="kernels workload: profiler-sized tensor-core cases")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-collapse", action="store_true", help="skip the deep-stack-collapse variant run")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

@@ -61,6 +61,7 @@ typedef struct hero_config {
   int dtype;               /* HERO_DTYPE_* */
   int has_gate;            /* 1: adaLN also yields a gate per branch (6 chunks instead of 4) */
   unsigned long long seed; /* low 32 bits seed the sampler's counter-based hash */
+  int deep_collapse;       /* 1: hero_step keeps ONE history pair for the whole deep stack (see below) */
 } hero_config;
 
 /* Device pointers to one block's parameters (borrowed for the context's lifetime).
@@ -133,6 +134,17 @@ int hero_refresh_block(hero_ctx *ctx, int block, void *d_x, const void *d_temb,
  * x += g_last + (g_last - g_prev) * k/d for the attention and the FFN history. */
 int hero_extrapolate_block(hero_ctx *ctx, int block, void *d_x, int k, int d);
 
+/* Deep-stack collapse (hero_config.deep_collapse = 1).  Eq. 5 is linear in the cached features and a
+ * deep block touches nothing but the residual stream, so the sum over deep blocks of their
+ * extrapolated branch outputs equals the extrapolation of the summed branch outputs.  With the flag
+ * set, a full step accumulates sum_l (G_attn^l + G_ffn^l) over the deep blocks in fp32 (two history
+ * slots for the whole stack instead of four tensors per deep block) and a cached step adds its
+ * extrapolation to x in one pass.  Same result in exact arithmetic, fewer roundings in bf16, about
+ * (n_deep * 4 - 2) fewer cache tensors.  In this mode the deep blocks are driven by hero_step only:
+ * hero_refresh_block and hero_extrapolate_block on a deep block return HERO_ERR_STATE, and
+ * hero_extrapolate_deep_stack applies the collapsed extrapolation on its own. */
+int hero_extrapolate_deep_stack(hero_ctx *ctx, void *d_x, int k, int d);
+
 /* One denoising step through all blocks with Algorithm 1's schedule: a full step when
  * step < warmup_full_steps or (step - (warmup-1)) % M == 0, else select+refresh in shallow
  * blocks and extrapolation in deep ones with k, d taken from the recorded full steps. */
@@ -198,6 +210,8 @@ int hero_isolated_status(void *stream);
 #define HERO_STATE_G_ATTN_PREV 6 /* deep blocks: g_prev */
 #define HERO_STATE_G_FFN_PREV  7
 #define HERO_STATE_STEPS    8   /* int32[3]: number of full steps seen, s_prev, s_last (block ignored) */
+#define HERO_STATE_STACK_LAST 9  /* deep_collapse: fp32 [B,N,D] sum of the deep blocks' branch outputs, latest full step */
+#define HERO_STATE_STACK_PREV 10 /* deep_collapse: the same for the full step before (block ignored for both) */
 /* Copy a piece of per-block state to / from host memory (synchronises the stream). */
 int hero_state_get(hero_ctx *ctx, int block, int what, void *h_out, long long bytes);
 int hero_state_set(hero_ctx *ctx, int block, int what, const void *h_in, long long bytes);

@@ -232,6 +232,16 @@ def extrapolate(g_prev, g_last, k: int, d: int):
     return g_last + (g_last - g_prev) * (F64(k) / F64(d))
 
 
+def extrapolate_stack(g_prev_list, g_last_list, k: int, d: int):
+    """Eq. 5 applied once to the SUM of several cached features (all branches of all deep
+    blocks).  Eq. 5 is linear in G and a deep block only adds its G to the residual stream
+    (Sec. 4.4), so this equals the sum of the per-block extrapolations; it is written out
+    separately so that the equality can be tested."""
+    s_prev = sum(np.asarray(g, F64) for g in g_prev_list)
+    s_last = sum(np.asarray(g, F64) for g in g_last_list)
+    return extrapolate(s_prev, s_last, k, d)
+
+
 # =============================================================================
 # Per-block state and the three block operations of Algorithm 1
 # =============================================================================
@@ -336,6 +346,14 @@ class HeroOracle:
         for i in range(2):
             prev = st.g_prev[i] if st.g_prev[i] is not None else st.g_last[i]   # one slot: Delta = 0
             x += extrapolate(prev, st.g_last[i], k, d)
+        return x
+
+    def deep_stack_extrapolate(self, x, k: int, d: int):
+        """All deep blocks of a cached step at once: x += Eq. 5 of the summed histories."""
+        deep = self.blocks[self.cfg.n_shallow:]
+        last = [st.g_last[i] for st in deep for i in range(2)]
+        prev = [(st.g_prev[i] if st.g_prev[i] is not None else st.g_last[i]) for st in deep for i in range(2)]
+        x += extrapolate_stack(prev, last, k, d)
         return x
 
     # ---- selection for one shallow block ----

@@ -16,14 +16,15 @@ LIB_PATH = os.path.join(_HERE, "libhero.so")
 
 OK, ERR_ARG, ERR_ALIGN, ERR_CAP, ERR_STATE, ERR_CUDA, ERR_TIMEOUT, ERR_NOMEM = 0, -1, -2, -3, -4, -5, -6, -7
 DTYPE_FP32, DTYPE_BF16 = 0, 1
-STATE = dict(ages=0, calls=1, k=2, v=3, g_attn=4, g_ffn=5, g_attn_prev=6, g_ffn_prev=7, steps=8)
+STATE = dict(ages=0, calls=1, k=2, v=3, g_attn=4, g_ffn=5, g_attn_prev=6, g_ffn_prev=7, steps=8, stack_last=9,
+             stack_prev=10)
 
 PROF_CATEGORIES = ("select", "modulation", "gather_ln", "gemm", "attention", "residual", "extrapolate")
 
 EXPORTS = [
     "hero_init", "hero_reset", "hero_destroy", "hero_strerror", "hero_check_status", "hero_last_cuda_error",
     "hero_device_bytes", "hero_launch_count", "hero_profile_begin", "hero_profile_end", "hero_select_tokens", "hero_next_n_sel", "hero_refresh_block",
-    "hero_extrapolate_block", "hero_step", "hero_step_host", "hero_is_full_step", "hero_extrapolate",
+    "hero_extrapolate_block", "hero_extrapolate_deep_stack", "hero_step", "hero_step_host", "hero_is_full_step", "hero_extrapolate",
     "hero_gather_rows", "hero_scatter_rows", "hero_gemm_bf16", "hero_attention_bf16", "hero_attention_bf16_static", "hero_isolated_status",
     "hero_state_get", "hero_state_set",
 ]
@@ -34,7 +35,7 @@ class HeroConfig(C.Structure):
         "n_blocks", "n_shallow", "hidden", "n_heads", "head_dim", "ffn_dim", "temb_dim",
         "batch", "frames", "grid_h", "grid_w", "n_text", "patch_h", "patch_w",
         "ratio_num", "ratio_den", "quota_mode", "warmup_full_steps", "full_interval", "dtype", "has_gate")
-    ] + [("seed", C.c_ulonglong)]
+    ] + [("seed", C.c_ulonglong), ("deep_collapse", C.c_int)]
 
 
 class HeroBlockWeights(C.Structure):
@@ -79,6 +80,7 @@ def load() -> C.CDLL:
         "hero_next_n_sel": (i, [vp, i]),
         "hero_refresh_block": (i, [vp, i, vp, vp, vp, i]),
         "hero_extrapolate_block": (i, [vp, i, vp, i, i]),
+        "hero_extrapolate_deep_stack": (i, [vp, vp, i, i]),
         "hero_step": (i, [vp, i, vp, vp]),
         "hero_step_host": (i, [vp, i, vp, vp]),
         "hero_is_full_step": (i, [vp, i]),
@@ -191,6 +193,9 @@ class Hero:
     def hero_extrapolate_block(self, block: int, x, k: int, d: int):
         _check(self.lib.hero_extrapolate_block(self.ctx, block, _ptr(x), k, d), "hero_extrapolate_block")
 
+    def hero_extrapolate_deep_stack(self, x, k: int, d: int):
+        _check(self.lib.hero_extrapolate_deep_stack(self.ctx, _ptr(x), k, d), "hero_extrapolate_deep_stack")
+
     def hero_step(self, step: int, x, temb):
         _check(self.lib.hero_step(self.ctx, step, _ptr(x), _ptr(temb)), "hero_step")
 
@@ -231,6 +236,8 @@ class Hero:
             return torch.empty(1, dtype=torch.int32)
         if what == "steps":
             return torch.empty(3, dtype=torch.int32)
+        if what in ("stack_last", "stack_prev"):
+            return torch.empty(self.cfg["batch"], self.N, self.cfg["hidden"], dtype=torch.float32)
         return torch.empty(self.cfg["batch"], self.N, self.cfg["hidden"], dtype=self.dt)
 
     def hero_state_get(self, block: int, what: str) -> torch.Tensor:

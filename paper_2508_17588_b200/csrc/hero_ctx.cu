@@ -42,6 +42,10 @@ struct hero_ctx {
   std::vector<hero_block_weights> w;
   std::vector<BlockMem> blk;
   void* kv_tmp[2] = {nullptr, nullptr};  // K/V of deep blocks during full passes (never cached)
+  // deep-stack collapse: branch outputs of a deep block are transient, their fp32 sum over the stack is kept
+  void* deep_g[2] = {nullptr, nullptr};
+  float* stack_hist[2] = {nullptr, nullptr};
+  int stack_last = 0, stack_n = 0, stack_new = 0;
   void *ws_a = nullptr, *ws_q = nullptr, *ws_o = nullptr, *ws_u = nullptr;
   float* mod = nullptr;                  // [B, n_mod*D] adaLN vectors of the current block
   int* idx_ws = nullptr;                 // [n_shallow, idx_cap] selection lists of the current step
@@ -162,7 +166,11 @@ int refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, const i
 
   void *kdst, *vdst, *ga, *gf;
   int new_slot = 0;
-  if (deep) {
+  const bool collapse = deep && g.deep_collapse;
+  if (collapse) {
+    kdst = c->kv_tmp[0]; vdst = c->kv_tmp[1];
+    ga = c->deep_g[0]; gf = c->deep_g[1];
+  } else if (deep) {
     new_slot = bm.n_hist == 0 ? 0 : (bm.last_slot ^ 1);
     kdst = c->kv_tmp[0]; vdst = c->kv_tmp[1];
     ga = bm.hist[0][new_slot]; gf = bm.hist[1][new_slot];
@@ -211,6 +219,11 @@ int refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, const i
   HERO_TRY(run_gemm(c, c->ws_u, w.w_2, w.b_2, M, D, F, o_dn));
 
   // x = (x + G_attn) + G_ffn for every row: fresh rows and cached rows alike
+  if (collapse) {
+    HERO_LAUNCH(c, HERO_PROF_RESIDUAL,
+                launch_residual2_acc(d_x, ga, gf, c->stack_hist[c->stack_new], c->elems, g.dtype, c->stream));
+    return HERO_OK;
+  }
   HERO_LAUNCH(c, HERO_PROF_RESIDUAL, launch_residual2(d_x, ga, gf, c->elems, g.dtype, c->stream));
 
   if (full) {
@@ -221,6 +234,15 @@ int refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, const i
       HERO_CUDA_TRY(cudaMemsetAsync(bm.ages[bm.ages_cur], 0, (size_t)c->n_video * sizeof(uint16_t), c->stream));
     }
   }
+  return HERO_OK;
+}
+
+int extrapolate_stack(hero_ctx* c, void* d_x, int k, int d) {
+  if (c->stack_n == 0) return HERO_ERR_STATE;
+  const int last = c->stack_last, prev = c->stack_n >= 2 ? (last ^ 1) : last;   // one slot only: Delta = 0
+  HERO_LAUNCH(c, HERO_PROF_EXTRAPOLATE,
+              launch_extrapolate_stack(d_x, c->stack_hist[prev], c->stack_hist[last], c->elems, k, d, c->cfg.dtype,
+                                       c->stream));
   return HERO_OK;
 }
 
@@ -245,6 +267,7 @@ int validate(const hero_config* g) {
   if (g->warmup_full_steps < 1 || g->full_interval < 0) return HERO_ERR_ARG;
   if (g->dtype != HERO_DTYPE_FP32 && g->dtype != HERO_DTYPE_BF16) return HERO_ERR_ARG;
   if (g->n_shallow > kMaxSelectBatch) return HERO_ERR_ARG;
+  if (g->deep_collapse != 0 && g->deep_collapse != 1) return HERO_ERR_ARG;
   if (g->dtype == HERO_DTYPE_BF16) {
     if (g->head_dim != 64 || g->hidden % 8 || g->ffn_dim % 8 || g->temb_dim % 8) return HERO_ERR_ALIGN;
   } else {
@@ -319,9 +342,14 @@ int hero_init(hero_ctx** out, const hero_config* cfg, const hero_block_weights* 
     if (l < cfg->n_shallow) {
       A(&bm.k, tensor); A(&bm.v, tensor); A(&bm.g[0], tensor); A(&bm.g[1], tensor);
       A((void**)&bm.ages[0], (size_t)c->n_video * 2); A((void**)&bm.ages[1], (size_t)c->n_video * 2);
-    } else {
+    } else if (!cfg->deep_collapse) {
       for (int br = 0; br < 2; ++br) for (int s = 0; s < 2; ++s) A(&bm.hist[br][s], tensor);
     }
+  }
+  if (cfg->deep_collapse && cfg->n_shallow < cfg->n_blocks) {
+    A(&c->deep_g[0], tensor); A(&c->deep_g[1], tensor);
+    A((void**)&c->stack_hist[0], (size_t)c->elems * sizeof(float));
+    A((void**)&c->stack_hist[1], (size_t)c->elems * sizeof(float));
   }
   if (cfg->n_shallow < cfg->n_blocks) { A(&c->kv_tmp[0], tensor); A(&c->kv_tmp[1], tensor); }
   A(&c->ws_a, tensor); A(&c->ws_q, tensor); A(&c->ws_o, tensor);
@@ -349,6 +377,7 @@ int hero_reset(hero_ctx* c) {
     if (bm.ages[1]) HERO_CUDA_TRY(cudaMemsetAsync(bm.ages[1], 0, (size_t)c->n_video * 2, c->stream));
   }
   c->n_full = 0; c->s_prev = 0; c->s_last = 0;
+  c->stack_last = 0; c->stack_n = 0; c->stack_new = 0;
   return HERO_OK;
 }
 
@@ -430,6 +459,7 @@ int hero_refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, co
     HERO_LAUNCH(c, HERO_PROF_RESIDUAL, launch_residual2(d_x, bm.g[0], bm.g[1], c->elems, c->cfg.dtype, c->stream));
     return HERO_OK;
   }
+  if (c->cfg.deep_collapse && block >= c->cfg.n_shallow) return HERO_ERR_STATE;   // driven by hero_step only
   if (d_idx == nullptr) {
     if (n_sel != c->N) return HERO_ERR_ARG;
   } else {
@@ -444,7 +474,15 @@ int hero_extrapolate_block(hero_ctx* c, int block, void* d_x, int k, int d) {
   if (block < c->cfg.n_shallow || block >= c->cfg.n_blocks) return HERO_ERR_ARG;
   if (k < 0 || d <= 0) return HERO_ERR_ARG;
   if (!aligned16(d_x)) return HERO_ERR_ALIGN;
+  if (c->cfg.deep_collapse) return HERO_ERR_STATE;          // no per-block history in this mode
   return extrapolate_block(c, block, d_x, k, d);
+}
+
+int hero_extrapolate_deep_stack(hero_ctx* c, void* d_x, int k, int d) {
+  if (!c || !d_x || k < 0 || d <= 0) return HERO_ERR_ARG;
+  if (!aligned16(d_x)) return HERO_ERR_ALIGN;
+  if (!c->cfg.deep_collapse || c->cfg.n_shallow >= c->cfg.n_blocks) return HERO_ERR_STATE;
+  return extrapolate_stack(c, d_x, k, d);
 }
 
 int hero_is_full_step(const hero_ctx* c, int step) {
@@ -456,8 +494,14 @@ int hero_step(hero_ctx* c, int step, void* d_x, const void* d_temb) {
   if (!c || !d_x || !d_temb || step < 0) return HERO_ERR_ARG;
   if (!aligned16(d_x) || !aligned16(d_temb)) return HERO_ERR_ALIGN;
   const hero_config& g = c->cfg;
+  const bool collapse = g.deep_collapse && g.n_shallow < g.n_blocks;
   if (is_full(g, step)) {
+    if (collapse) {                          // the deep stack's branch outputs are summed into a fresh slot
+      c->stack_new = c->stack_n == 0 ? 0 : (c->stack_last ^ 1);
+      HERO_CUDA_TRY(cudaMemsetAsync(c->stack_hist[c->stack_new], 0, (size_t)c->elems * sizeof(float), c->stream));
+    }
     for (int l = 0; l < g.n_blocks; ++l) HERO_TRY(refresh_block(c, l, d_x, d_temb, nullptr, c->N));
+    if (collapse) { c->stack_last = c->stack_new; if (c->stack_n < 2) c->stack_n++; }
     c->s_prev = c->s_last; c->s_last = step; c->n_full++;
     return HERO_OK;
   }
@@ -488,6 +532,9 @@ int hero_step(hero_ctx* c, int step, void* d_x, const void* d_temb) {
         HERO_LAUNCH(c, HERO_PROF_RESIDUAL,
                     launch_residual2(d_x, c->blk[l].g[0], c->blk[l].g[1], c->elems, g.dtype, c->stream));
       }
+    } else if (collapse) {
+      HERO_TRY(extrapolate_stack(c, d_x, k, d));   // Eq. 5 once, on the sums over all deep blocks
+      break;
     } else {
       HERO_TRY(extrapolate_block(c, l, d_x, k, d));
     }
@@ -587,10 +634,17 @@ int hero_isolated_status(void* stream) { return poll_isolated_status((cudaStream
 static int state_ptr(hero_ctx* c, int block, int what, void** p, size_t* bytes) {
   const hero_config& g = c->cfg;
   if (what == HERO_STATE_STEPS) { *p = nullptr; *bytes = 12; return HERO_OK; }
+  if (what == HERO_STATE_STACK_LAST || what == HERO_STATE_STACK_PREV) {
+    if (!g.deep_collapse || !c->stack_hist[0]) return HERO_ERR_ARG;
+    *p = c->stack_hist[what == HERO_STATE_STACK_LAST ? c->stack_last : (c->stack_last ^ 1)];
+    *bytes = (size_t)c->elems * sizeof(float);
+    return HERO_OK;
+  }
   if (block < 0 || block >= g.n_blocks) return HERO_ERR_ARG;
   BlockMem& bm = c->blk[block];
   const bool deep = block >= g.n_shallow;
   const size_t tensor = (size_t)c->elems * c->esz;
+  if (deep && g.deep_collapse) return HERO_ERR_ARG;        // deep blocks keep no per-block state in this mode
   switch (what) {
     case HERO_STATE_AGES: if (deep) return HERO_ERR_ARG; *p = bm.ages[bm.ages_cur]; *bytes = (size_t)c->n_video * 2; return HERO_OK;
     case HERO_STATE_CALLS: *p = nullptr; *bytes = 4; return HERO_OK;
@@ -630,6 +684,8 @@ int hero_state_set(hero_ctx* c, int block, int what, const void* h_in, long long
   if (what == HERO_STATE_CALLS) { int v; memcpy(&v, h_in, 4); if (v < 0) return HERO_ERR_ARG; c->blk[block].calls = v; return HERO_OK; }
   HERO_CUDA_TRY(cudaMemcpyAsync(p, h_in, need, cudaMemcpyHostToDevice, c->stream));
   HERO_CUDA_TRY(cudaStreamSynchronize(c->stream));
+  if (what == HERO_STATE_STACK_LAST) { if (c->stack_n < 1) c->stack_n = 1; return HERO_OK; }
+  if (what == HERO_STATE_STACK_PREV) { c->stack_n = 2; return HERO_OK; }
   if (block >= c->cfg.n_shallow) {   // planting a deep block's history marks the slots as valid
     BlockMem& bm = c->blk[block];
     if (what == HERO_STATE_G_ATTN || what == HERO_STATE_G_FFN) { if (bm.n_hist < 1) bm.n_hist = 1; }

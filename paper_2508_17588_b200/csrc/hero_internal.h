@@ -80,6 +80,10 @@ int launch_extrapolate_residual(void* x, const void* ga_prev, const void* ga_las
                                 const void* gf_last, long long n, int k, int d, int dtype, cudaStream_t s);
 // x = (x + ga) + gf
 int launch_residual2(void* x, const void* ga, const void* gf, long long n, int dtype, cudaStream_t s);
+// deep-stack collapse: x = (x + ga) + gf, acc += ga + gf (fp32);  x += s_last + (s_last - s_prev) * k/d
+int launch_residual2_acc(void* x, const void* ga, const void* gf, float* acc, long long n, int dtype, cudaStream_t s);
+int launch_extrapolate_stack(void* x, const float* s_prev, const float* s_last, long long n, int k, int d, int dtype,
+                             cudaStream_t s);
 int launch_gather_rows(const void* src, const int* idx, void* dst, int B, int N, int n_sel, int D,
                        int dtype, cudaStream_t s);
 int launch_scatter_rows(const void* src, const int* idx, void* dst, int B, int N, int n_sel, int D,

@@ -201,6 +201,92 @@ __global__ void __launch_bounds__(kStreamThreads) residual2_kernel(T* __restrict
   }
 }
 
+// ------------------------------------------------------------------ deep-stack collapse
+// fp32 side-band packets matching one 16-byte packet of T
+template <typename T>
+struct AccVec;
+template <>
+struct AccVec<float> {
+  __device__ static void load(const float* p, long long i, float (&f)[4]) {
+    const float4 v = __ldcs(reinterpret_cast<const float4*>(p) + i);
+    f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;
+  }
+  __device__ static void store(float* p, long long i, const float (&f)[4]) {
+    __stcs(reinterpret_cast<float4*>(p) + i, make_float4(f[0], f[1], f[2], f[3]));
+  }
+};
+template <>
+struct AccVec<__nv_bfloat16> {
+  __device__ static void load(const float* p, long long i, float (&f)[8]) {
+    const float4 a = __ldcs(reinterpret_cast<const float4*>(p) + 2 * i), b = __ldcs(reinterpret_cast<const float4*>(p) + 2 * i + 1);
+    f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
+  }
+  __device__ static void store(float* p, long long i, const float (&f)[8]) {
+    __stcs(reinterpret_cast<float4*>(p) + 2 * i, make_float4(f[0], f[1], f[2], f[3]));
+    __stcs(reinterpret_cast<float4*>(p) + 2 * i + 1, make_float4(f[4], f[5], f[6], f[7]));
+  }
+};
+
+// Full step, deep block, collapse mode: x = (x + ga) + gf and acc += ga + gf (fp32 running sum of the
+// deep stack's branch outputs, the quantity Eq. 5 is applied to on cached steps).
+template <typename T>
+__global__ void __launch_bounds__(kStreamThreads) residual2_acc_kernel(T* __restrict__ x, const T* __restrict__ ga,
+                                                                       const T* __restrict__ gf,
+                                                                       float* __restrict__ acc, long long n) {
+  using V = Vec<T>;
+  const long long n_vec = n / V::N;
+  V* xv = reinterpret_cast<V*>(x);
+  const V* a = reinterpret_cast<const V*>(ga);
+  const V* f = reinterpret_cast<const V*>(gf);
+  const long long stride = (long long)gridDim.x * kStreamThreads;
+  for (long long i = (long long)blockIdx.x * kStreamThreads + threadIdx.x; i < n_vec; i += stride) {
+    const V vx = ld_stream(xv + i), va = ld_stream(a + i), vf = ld_stream(f + i);
+    float fx[V::N], fa[V::N], ff[V::N], fs[V::N];
+    vx.unpack(fx); va.unpack(fa); vf.unpack(ff);
+    AccVec<T>::load(acc, i, fs);
+#pragma unroll
+    for (int j = 0; j < V::N; ++j) { fx[j] = (fx[j] + fa[j]) + ff[j]; fs[j] += fa[j] + ff[j]; }
+    V r; r.pack(fx);
+    st_stream(xv + i, r);
+    AccVec<T>::store(acc, i, fs);
+  }
+  const long long tail0 = n_vec * V::N;
+  if (blockIdx.x == 0 && threadIdx.x < n - tail0) {
+    const long long i = tail0 + threadIdx.x;
+    const float va = to_f(ga[i]), vf = to_f(gf[i]);
+    x[i] = from_f<T>((to_f(x[i]) + va) + vf);
+    acc[i] += va + vf;
+  }
+}
+
+// Cached step, whole deep stack in one pass: x += s_last + (s_last - s_prev) * c  (Eq. 5 on the sums).
+template <typename T>
+__global__ void __launch_bounds__(kStreamThreads) extrapolate_stack_kernel(T* __restrict__ x,
+                                                                           const float* __restrict__ s_prev,
+                                                                           const float* __restrict__ s_last,
+                                                                           long long n, float c) {
+  using V = Vec<T>;
+  const long long n_vec = n / V::N;
+  V* xv = reinterpret_cast<V*>(x);
+  const long long stride = (long long)gridDim.x * kStreamThreads;
+  for (long long i = (long long)blockIdx.x * kStreamThreads + threadIdx.x; i < n_vec; i += stride) {
+    const V vx = ld_stream(xv + i);
+    float fx[V::N], fp[V::N], fl[V::N];
+    vx.unpack(fx);
+    AccVec<T>::load(s_prev, i, fp);
+    AccVec<T>::load(s_last, i, fl);
+#pragma unroll
+    for (int j = 0; j < V::N; ++j) fx[j] += fmaf(fl[j] - fp[j], c, fl[j]);
+    V r; r.pack(fx);
+    st_stream(xv + i, r);
+  }
+  const long long tail0 = n_vec * V::N;
+  if (blockIdx.x == 0 && threadIdx.x < n - tail0) {
+    const long long i = tail0 + threadIdx.x;
+    x[i] = from_f<T>(to_f(x[i]) + fmaf(s_last[i] - s_prev[i], c, s_last[i]));
+  }
+}
+
 // ------------------------------------------------------------------ gather / scatter of rows
 // One warp moves one row in 16-byte packets, four packets per lane in flight at a time (2 KB per
 // warp, 16 KB per CTA); GATHER reads row idx[i] and writes row i, SCATTER the reverse.  Rows not
@@ -467,6 +553,37 @@ int launch_residual2(void* x, const void* ga, const void* gf, long long n, int d
   } else {
     residual2_kernel<float><<<stream_grid(n / 4), kStreamThreads, 0, s>>>((float*)x, (const float*)ga,
                                                                            (const float*)gf, n);
+  }
+  HERO_CUDA_TRY(cudaGetLastError());
+  return HERO_OK;
+}
+
+static int wide_grid(long long n_vec) {
+  long long blocks = (n_vec + kStreamThreads - 1) / kStreamThreads;
+  const long long cap = (long long)num_sms() * 32;
+  return (int)(blocks < 1 ? 1 : (blocks > cap ? cap : blocks));
+}
+
+int launch_residual2_acc(void* x, const void* ga, const void* gf, float* acc, long long n, int dtype, cudaStream_t s) {
+  if (dtype == HERO_DTYPE_BF16) {
+    using T = __nv_bfloat16;
+    residual2_acc_kernel<T><<<wide_grid(n / Vec<T>::N), kStreamThreads, 0, s>>>((T*)x, (const T*)ga, (const T*)gf, acc, n);
+  } else {
+    residual2_acc_kernel<float><<<wide_grid(n / 4), kStreamThreads, 0, s>>>((float*)x, (const float*)ga,
+                                                                          (const float*)gf, acc, n);
+  }
+  HERO_CUDA_TRY(cudaGetLastError());
+  return HERO_OK;
+}
+
+int launch_extrapolate_stack(void* x, const float* s_prev, const float* s_last, long long n, int k, int d, int dtype,
+                             cudaStream_t s) {
+  const float c = (float)k / (float)d;
+  if (dtype == HERO_DTYPE_BF16) {
+    using T = __nv_bfloat16;
+    extrapolate_stack_kernel<T><<<wide_grid(n / Vec<T>::N), kStreamThreads, 0, s>>>((T*)x, s_prev, s_last, n, c);
+  } else {
+    extrapolate_stack_kernel<float><<<wide_grid(n / 4), kStreamThreads, 0, s>>>((float*)x, s_prev, s_last, n, c);
   }
   HERO_CUDA_TRY(cudaGetLastError());
   return HERO_OK;

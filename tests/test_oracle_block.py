@@ -294,3 +294,34 @@ def test_tiny_config_ten_steps_runs_and_follows_schedule():
     assert orc.blocks[0].calls == 8 and orc.blocks[1].calls == 8
     assert orc.blocks[2].calls == 0
     assert O.n_selected(cfg, 0) == 32           # 25 % of 128 video tokens
+
+
+# ---------------------------------------------------------------- deep-stack collapse (linearity of Eq. 5)
+def test_extrapolating_the_sum_equals_summing_the_extrapolations():
+    rng = np.random.default_rng(5)
+    prev = [rng.standard_normal((2, 7, 16)) for _ in range(6)]
+    last = [p + 0.1 * rng.standard_normal(p.shape) for p in prev]
+    for k, d in ((1, 1), (2, 5), (4, 5), (0, 3)):
+        one_by_one = sum(O.extrapolate(p, l, k, d) for p, l in zip(prev, last))
+        assert np.allclose(O.extrapolate_stack(prev, last, k, d), one_by_one, rtol=0, atol=1e-12)
+    # not a tautology: a non-linear rule (e.g. clipping each block's step) would break it
+    clipped = sum(np.clip(O.extrapolate(p, l, 4, 5), -0.5, 0.5) for p, l in zip(prev, last))
+    assert not np.allclose(np.clip(O.extrapolate_stack(prev, last, 4, 5), -0.5, 0.5), clipped)
+
+
+def test_deep_stack_extrapolate_matches_block_by_block_step():
+    cfgd = dict(S.CONFIGS["tiny"], n_blocks=5, n_shallow=1, full_interval=3)
+    weights = [S.block_weights(cfgd, l) for l in range(cfgd["n_blocks"])]
+    a = O.HeroOracle(O.Config.from_dict(cfgd), weights)
+    x0 = S.tokens(cfgd)
+    for s in range(3):                                    # full at 0, 1; cached at 2
+        xa = a.step(s, x0, S.temb(cfgd, s))
+    # redo the cached step's deep part with the collapsed form on a copy of the state before it
+    b = O.HeroOracle(O.Config.from_dict(cfgd), weights)
+    for s in range(2):
+        b.step(s, x0, S.temb(cfgd, s))
+    xb = np.array(x0, np.float64)
+    rows = b.select(0)
+    b.block_refresh(0, xb, S.temb(cfgd, 2), rows)
+    b.deep_stack_extrapolate(xb, 1, 1)
+    assert np.allclose(xa, xb, rtol=0, atol=1e-11)
