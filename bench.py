@@ -8,7 +8,7 @@ into the caches, residual adds, and linear extrapolation in the deep blocks.  Th
 full steps that fill the caches are set-up, not timed; a full step is timed once and reported
 in `config` together with the 50-step schedule average.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl hero|reference] [--workload dit42|aether|tiny|kernels [--only LIST] [--small]]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl hero|reference] [--workload dit42|aether|paper_hp|tiny|kernels [--only LIST] [--small]]
 
 Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank runs its own sequence on its
 own GPU (independent problems, no data-path collective): "scaling": "weak".
@@ -541,7 +541,7 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="hero", choices=["hero", "reference"])
-    ap.add_argument("--workload", default="dit42", choices=["dit42", "aether", "tiny", "kernels"])
+    ap.add_argument("--workload", default="dit42", choices=["dit42", "aether", "paper_hp", "tiny", "kernels"])
     ap.add_argument("--only", default="", help="kernels workload: comma list of select,extrapolate,gather,scatter,"
                                                "attention,gemm,block")
     ap.add_argument("--small", action="store_true", help="kernels workload: profiler-sized tensor-core cases")

@@ -148,3 +148,28 @@ def test_call_order_and_argument_errors():
         hero.hero_refresh_block(0, x[:, :, 1:], t)    # misaligned view
     assert e.value.code == -2
     hero.close()
+
+
+def test_paper_hyperparameters_small_model():
+    """The paper's own setting in miniature: 2x3 patches, R = 0.2 with round-half-up quotas (one token per
+    full patch), three of four blocks refreshed, a full step every M = 2 steps; 9 steps through hero_step."""
+    cfgd = dict(S.CONFIGS["tiny"], frames=2, grid_h=6, grid_w=9, patch_h=2, patch_w=3, ratio_num=1, ratio_den=5,
+                quota_mode=1, n_shallow=3, full_interval=2, steps=9, seed=77)
+    orc, hero, _ = make_pair(cfgd)
+    cfg = O.Config.from_dict(cfgd)
+    assert O.n_selected(cfg, 0) == cfg.n_video // 6
+    x_host = S.tokens(cfgd)
+    n_full = 0
+    for s in range(cfgd["steps"]):                       # full at 0, 1, 3, 5, 7; cached at 2, 4, 6, 8
+        temb = S.temb(cfgd, s)
+        want = orc.step(s, x_host, temb)
+        x = to_dev(x_host, "fp32")
+        assert hero.hero_is_full_step(s) == orc.is_full_step(s)
+        n_full += orc.is_full_step(s)
+        hero.hero_step(s, x, to_dev(temb, "fp32"))
+        assert rel_l2(to_host(x), want) <= FP32_TOL, s
+        for l in range(cfgd["n_shallow"]):
+            assert np.array_equal(hero.hero_state_get(l, "ages").numpy(), orc.blocks[l].ages)
+            assert int(hero.hero_state_get(l, "calls")[0]) == orc.blocks[l].calls
+    assert n_full == 5
+    hero.close()

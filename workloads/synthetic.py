@@ -48,6 +48,10 @@ CONFIGS = {
     # config 5: Aether-shaped sequence, 17 latent frames, 48 latent channels
     "aether": dict(_COGVIDEO, n_blocks=42, n_shallow=14, frames=17, ratio_num=1, ratio_den=4,
                    full_interval=5, seed=4, steps=50, latent_channels=48),
+    # the paper's own hyper-parameters (Sec. 5.1): 2x3 patches, R = 0.2 rounded per patch (Table 3 implies
+    # round(6R) tokens), the first 20 blocks refreshed, a full step every M = 2 steps, 11 latent frames
+    "paper_hp": dict(_COGVIDEO, n_blocks=42, n_shallow=20, frames=11, patch_h=2, patch_w=3, ratio_num=1,
+                     ratio_den=5, quota_mode=1, full_interval=2, seed=5, steps=50),
 }
 
 
