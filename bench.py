@@ -166,6 +166,13 @@ def cpu_cores_used():
         return os.cpu_count() or 1
 
 
+def workload_config(args, cfg) -> dict:
+    """The part of `config` that names the workload; both arms print the same keys."""
+    return {"workload": args.workload, "blocks": cfg["n_blocks"], "refresh_blocks": cfg["n_shallow"],
+            "refresh_ratio": cfg["ratio_num"] / cfg["ratio_den"], "batch": cfg["batch"],
+            "tokens_per_seq": S.n_rows(cfg), "hidden": cfg["hidden"]}
+
+
 def run_reference(args, cfg, rank, world):
     """Reference arm: the oracle on this machine's host cores, on bounded samples of the same workload."""
     if rank != 0:
@@ -178,12 +185,12 @@ def run_reference(args, cfg, rank, world):
         if i >= args.warmup:
             vals.append(sec)
     sec = statistics.mean(vals)
-    sample = ("per step: one shallow block refreshed on its 25 % selection (K/V of every selected row, branch "
+    sample = ("per step: one shallow block refreshed on its real selection (K/V of every selected row, branch "
               "outputs of 128 rows, scaled to all) + one deep block extrapolated, scaled by block counts")
     line = {"impl": "reference", "metric": METRIC, "value": tokens / sec, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": args.workload, "note": "oracle (numpy float64) timed on host cores"},
+            "config": dict(workload_config(args, cfg), note="oracle (numpy float64) timed on host cores"),
             "cpu_baseline": {"value": tokens / sec, "unit": UNIT, "cores": cpu_cores_used(), "kind": "oracle",
                              "sample": sample},
             "e2e": {"value": tokens / sec, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
@@ -383,12 +390,11 @@ def run_hero(args, cfg, rank, world, local_rank):
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": cfg["dtype"], "data": "synthetic",
-                "config": {"workload": args.workload, "blocks": cfg["n_blocks"], "refresh_blocks": cfg["n_shallow"],
-                           "refresh_ratio": cfg["ratio_num"] / cfg["ratio_den"], "batch": B, "tokens_per_seq": N,
-                           "hidden": D, "l2": "inputs larger than L2 (each step streams > 30 GB of caches)",
-                           "full_step_ms": full_ms, "schedule_avg_ms_per_step": sched_ms,
-                           "schedule": "%d full + %d cached of %d steps" % (n_full, cfg["steps"] - n_full, cfg["steps"]),
-                           "device_bytes": mem, "parallelism": "replicas" if world > 1 else "single"},
+                "config": dict(workload_config(args, cfg),
+                               l2="inputs larger than L2 (each step streams > 30 GB of caches)",
+                               full_step_ms=full_ms, schedule_avg_ms_per_step=sched_ms,
+                               schedule="%d full + %d cached of %d steps" % (n_full, cfg["steps"] - n_full, cfg["steps"]),
+                               device_bytes=mem, parallelism="replicas" if world > 1 else "single"),
                 "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "breakdown_ms": breakdown}
         if collapsed:
             line["deep_collapse_variant"] = collapsed

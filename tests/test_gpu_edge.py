@@ -1,0 +1,142 @@
+"""GPU edge cases of the cached step through the C ABI: empty and full selections, ragged grids,
+no text rows, gates, context reuse, call-order and argument errors with a live context."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import hero_oracle as O
+from workloads import synthetic as S
+from tests.util import make_pair, rel_l2, to_dev, to_host
+
+pytestmark = pytest.mark.gpu
+
+FP32_TOL = 2e-5
+
+
+def H():
+    import paper_2508_17588_b200 as h
+    return h
+
+
+def _run_steps(cfgd, steps, dtype_tol):
+    orc, hero, _ = make_pair(cfgd)
+    x_host = S.tokens(cfgd)
+    outs = []
+    for s in range(steps):
+        temb = S.temb(cfgd, s)
+        want = orc.step(s, x_host, temb)
+        x = to_dev(x_host, cfgd["dtype"])
+        hero.hero_step(s, x, to_dev(temb, cfgd["dtype"]))
+        hero.hero_check_status()
+        assert rel_l2(to_host(x), want) <= dtype_tol, s
+        for l in range(cfgd["n_shallow"]):
+            assert np.array_equal(hero.hero_state_get(l, "ages").numpy(), orc.blocks[l].ages)
+        outs.append(x.clone())
+    return orc, hero, outs
+
+
+def test_selection_lists_that_are_sometimes_empty():
+    """R = 1/50 on a 2x3x3 grid with 2x2 patches: most calls select nothing, some one token."""
+    cfgd = dict(S.CONFIGS["tiny"], frames=2, grid_h=3, grid_w=3, n_text=3, ratio_num=1, ratio_den=50, steps=12, seed=5)
+    cfg = O.Config.from_dict(cfgd)
+    lens = [O.n_selected(cfg, c) for c in range(10)]
+    assert 0 in lens and max(lens) >= 1
+    _, hero, _ = _run_steps(cfgd, 12, FP32_TOL)
+    hero.close()
+
+
+def test_ratio_one_refreshes_every_video_row_bf16():
+    cfgd = dict(n_blocks=2, n_shallow=1, hidden=128, n_heads=2, head_dim=64, ffn_dim=256, temb_dim=64, batch=1,
+                frames=2, grid_h=5, grid_w=7, n_text=0, patch_h=2, patch_w=3, ratio_num=1, ratio_den=1,
+                quota_mode=1, warmup_full_steps=2, full_interval=0, dtype="bf16", has_gate=1, seed=8, steps=4)
+    cfg = O.Config.from_dict(cfgd)
+    assert O.n_selected(cfg, 0) == cfg.n_video == cfg.n_rows          # no text rows, clipped edge patches
+    weights = [S.block_weights(cfgd, l) for l in range(2)]
+    orc, hero, _ = make_pair(cfgd, weights)
+    x_host = S.tokens(cfgd)
+    for s in range(4):
+        temb = S.temb(cfgd, s)
+        want = orc.step(s, x_host, temb)
+        x = to_dev(x_host, "bf16")
+        hero.hero_step(s, x, to_dev(temb, "bf16"))
+        hero.hero_check_status()
+        assert rel_l2(to_host(x), want) <= 2e-2, s
+        st = orc.blocks[0]
+        for name, ref in (("k", st.k_cache), ("v", st.v_cache), ("g_attn", st.g[0]), ("g_ffn", st.g[1])):
+            ref[...] = to_host(hero.hero_state_get(0, name))             # teacher forcing
+    hero.close()
+
+
+def test_batch_three_with_gates_fp32():
+    cfgd = dict(S.CONFIGS["tiny"], batch=3, has_gate=1, frames=1, grid_h=7, grid_w=5, n_text=1, steps=5, seed=13)
+    _, hero, _ = _run_steps(cfgd, 5, FP32_TOL)
+    hero.close()
+
+
+def test_reset_reproduces_the_run_bit_for_bit_and_contexts_are_independent():
+    cfgd = dict(S.CONFIGS["tiny"], steps=5)
+    _, hero, first = _run_steps(cfgd, 5, FP32_TOL)
+    _, other, _ = make_pair(cfgd)                                      # a second live context on the same weights' values
+    hero.hero_reset()
+    x_host = S.tokens(cfgd)
+    for s in range(5):
+        t = to_dev(S.temb(cfgd, s), "fp32")
+        x, y = to_dev(x_host, "fp32"), to_dev(x_host, "fp32")
+        hero.hero_step(s, x, t)
+        other.hero_step(s, y, t)
+        assert torch.equal(x, first[s]) and torch.equal(y, first[s]), s
+    hero.close(); other.close()
+
+
+def test_call_order_and_argument_errors_with_a_live_context():
+    h = H()
+    cfgd = dict(S.CONFIGS["tiny"])
+    _, hero, _ = make_pair(cfgd)
+    cfg = O.Config.from_dict(cfgd)
+    x = to_dev(S.tokens(cfgd), "fp32")
+    t = to_dev(S.temb(cfgd, 0), "fp32")
+    idx = torch.zeros(cfg.n_video, dtype=torch.int32, device="cuda")
+
+    def code(fn):
+        with pytest.raises(h.HeroError) as e:
+            fn()
+        return e.value.code
+
+    assert code(lambda: hero.hero_step(2, x, t)) == -4                                  # cached step before any full step
+    assert code(lambda: hero.hero_extrapolate_block(2, x, 1, 1)) == -4                  # no history yet
+    assert code(lambda: hero.hero_extrapolate_block(0, x, 1, 1)) == -1                  # block 0 is a refresh block
+    assert code(lambda: hero.hero_extrapolate_block(2, x, 1, 0)) == -1                  # d = 0
+    assert code(lambda: hero.hero_refresh_block(9, x, t)) == -1                         # no such block
+    assert code(lambda: hero.hero_refresh_block(0, x, t, idx, cfg.n_rows + 1)) == -1    # list longer than the sequence
+    assert code(lambda: hero.hero_refresh_block(3, x, t, idx, 4)) == -1                 # partial refresh of a deep block
+    assert code(lambda: hero.hero_select_tokens(2, idx)) == -1                          # selection on a deep block
+    assert code(lambda: hero.hero_select_tokens(0, idx[:3])) == -3                      # capacity
+    misaligned = torch.zeros(x.numel() + 1, device="cuda")[1:].view_as(x)
+    assert code(lambda: hero.hero_step(0, misaligned, t)) == -2
+    # none of the refused calls changed any state: the run still matches a fresh context
+    _, fresh, _ = make_pair(cfgd)
+    for s in range(3):
+        ts = to_dev(S.temb(cfgd, s), "fp32")
+        a, b = to_dev(S.tokens(cfgd), "fp32"), to_dev(S.tokens(cfgd), "fp32")
+        hero.hero_step(s, a, ts)
+        fresh.hero_step(s, b, ts)
+        assert torch.equal(a, b)
+    assert int(hero.hero_state_get(0, "calls")[0]) == 1
+    hero.close(); fresh.close()
+
+
+def test_many_contexts_do_not_leak_device_memory():
+    cfgd = dict(S.CONFIGS["tiny"])
+    _, hero, w = make_pair(cfgd)
+    hero.close()
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+    for _ in range(20):
+        _, hero, _ = make_pair(cfgd, w)
+        x = to_dev(S.tokens(cfgd), "fp32")
+        hero.hero_step(0, x, to_dev(S.temb(cfgd, 0), "fp32"))
+        hero.close()
+        del x
+    torch.cuda.synchronize()
+    torch.cuda.empty_cache()
+    assert torch.cuda.mem_get_info()[0] >= free0 - (8 << 20)
