@@ -339,28 +339,28 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           tmem_st16(t_buf + ch * 16, *reinterpret_cast<uint32_t(*)[16]>(&packed[ch * 16]));
       }
       l_run = fmaf(l_run, alpha, sum);
-      if (j > 0) {
-        // P V of the previous tile was issued a whole iteration ago; observe its completion (every
-        // phase of the barrier is consumed) and, in the rare case the maximum moved, scale the
-        // accumulator down before this tile's product is added to it
+      if (j > 0 && grow) {
+        // Rare (warp-uniform): the maximum moved, so the accumulator is scaled down before this tile's
+        // product is added to it - once P V of tile j-1 has completed.  pv_full is only looked at here and
+        // at the very end, yet the parity wait is unambiguous: S of tile j was issued after P V of tile j-2
+        // (so that one is complete) and P V of tile j cannot start before this warp's arrival below, hence
+        // the barrier has completed either j-1 or j phases and "phase j-1 complete" is exactly the question.
         ok = mbar_wait(&pv_full[t], (j - 1) & 1, abort_flag);
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
-        if (grow) {                                    // warp-uniform; alpha is 1 for rows that did not move
-          tc_fence_after();
-          const float2 a2 = make_float2(alpha, alpha);
+        tc_fence_after();
+        const float2 a2 = make_float2(alpha, alpha);     // alpha is 1 for rows that did not move
 #pragma unroll
-          for (int ch = 0; ch < kHD / 16; ++ch) {
-            uint32_t r[16];
-            tmem_ld16(lane_base + kColO + ch * 16, r);
-            tmem_ld_wait();
+        for (int ch = 0; ch < kHD / 16; ++ch) {
+          uint32_t r[16];
+          tmem_ld16(lane_base + kColO + ch * 16, r);
+          tmem_ld_wait();
 #pragma unroll
-            for (int i = 0; i < 16; i += 2) {
-              const float2 v = __fmul2_rn(f2(r[i], r[i + 1]), a2);
-              r[i] = __float_as_uint(v.x); r[i + 1] = __float_as_uint(v.y);
-            }
-            tmem_st16(lane_base + kColO + ch * 16, r);
+          for (int i = 0; i < 16; i += 2) {
+            const float2 v = __fmul2_rn(f2(r[i], r[i + 1]), a2);
+            r[i] = __float_as_uint(v.x); r[i + 1] = __float_as_uint(v.y);
           }
+          tmem_st16(lane_base + kColO + ch * 16, r);
         }
       }
       tmem_st_wait();
