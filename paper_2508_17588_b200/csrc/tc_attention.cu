@@ -314,8 +314,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     float m_used = -INFINITY, l_run = 0.f;
     bool ok = true;
     for (int j = 0; j < n_kv; ++j) {
-      ok = mbar_wait(&s_full[t * 2 + (j & 1)], (j >> 1) & 1, abort_flag);
-      ok = __all_sync(0xFFFFFFFFu, ok);
+      ok = mbar_wait_warp(&s_full[t * 2 + (j & 1)], (j >> 1) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
       const uint32_t t_buf = lane_base + (uint32_t)(j & 1) * kKT;
@@ -345,8 +344,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         // at the very end, yet the parity wait is unambiguous: S of tile j was issued after P V of tile j-2
         // (so that one is complete) and P V of tile j cannot start before this warp's arrival below, hence
         // the barrier has completed either j-1 or j phases and "phase j-1 complete" is exactly the question.
-        ok = mbar_wait(&pv_full[t], (j - 1) & 1, abort_flag);
-        ok = __all_sync(0xFFFFFFFFu, ok);
+        ok = mbar_wait_warp(&pv_full[t], (j - 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
         const float2 a2 = make_float2(alpha, alpha);     // alpha is 1 for rows that did not move
@@ -368,10 +366,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       __syncwarp();
       if (lane == 0) mbar_arrive(&p_full[t * 2 + (j & 1)]);
     }
-    if (ok) {
-      ok = mbar_wait(&pv_full[t], (n_kv - 1) & 1, abort_flag);
-      ok = __all_sync(0xFFFFFFFFu, ok);
-    }
+    if (ok) ok = mbar_wait_warp(&pv_full[t], (n_kv - 1) & 1, abort_flag);
     if (ok) {
       tc_fence_after();
       const int qi = (qg * kQTiles + t) * kQT + quad * 32 + lane;

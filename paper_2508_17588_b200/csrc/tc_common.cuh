@@ -68,6 +68,14 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     if (mbar_try_wait(bar, parity)) return true;
   return mbar_wait_slow(bar, parity, abort_flag);
 }
+// The same wait for a whole converged warp whose lanes all poll the same barrier: one poll is one
+// warp-wide instruction, so the fast path is uniform by construction and only the slow path (where a lane
+// might give up a poll earlier than another) pays for a vote.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t it = 0; it < kWaitFastPolls; ++it)
+    if (mbar_try_wait(bar, parity)) return true;
+  return __all_sync(0xFFFFFFFFu, mbar_wait_slow(bar, parity, abort_flag));
+}
 // The same bounded wait for single-thread roles (TMA producer, MMA issuer) that sit beside busy
 // compute warps: it sleeps between polls from the start, so that the spinning thread does not
 // take issue slots and shared-memory bandwidth from the warps it is waiting for.
