@@ -513,6 +513,25 @@ def run_kernels(args):
             H.hero_isolated_status()
             tensor(f"gemm_{name}_m{M}", ms, 2 * M * n_out * kk)
             del a, w_, bias, c
+    if want("deep") and not args.small:
+        # the fused passes that only exist inside a context: Eq. 5 + residual of a deep block (12 B per
+        # element: 5 reads + 1 write) and the double residual add of a refresh block (8 B per element)
+        dcfg = dict(S.CONFIGS["block"], n_blocks=2, n_shallow=1)
+        weights = build_device_weights(dcfg, dev)
+        hero = H.Hero(dcfg, weights)
+        x = S.device_normal(dcfg["seed"], "x0", (B, N, D), 1.0, 0, None, dev).to(bf)
+        temb = S.device_normal(dcfg["seed"], "temb", (B, dcfg["temb_dim"]), 1.0, 0, None, dev).to(bf)
+        for s_ in range(2):
+            hero.hero_step(s_, x, temb)
+        n_el = B * N * D
+        hbm("extrapolate_residual_block", _time_flushed(lambda: hero.hero_extrapolate_block(1, x, 1, 1), iters, warm, flush),
+            12 * n_el)
+        idx0 = torch.zeros(1, dtype=torch.int32, device=dev)
+        hbm("residual2_block", _time_flushed(lambda: hero.hero_refresh_block(0, x, temb, idx0, 0), iters, warm, flush),
+            8 * n_el)
+        hero.hero_check_status()
+        hero.close()
+        del weights, x
     if want("block") and not args.small:
         bcfg = dict(S.CONFIGS["block"])
         weights = build_device_weights(bcfg, dev)
@@ -549,7 +568,7 @@ def main():
     ap.add_argument("--impl", default="hero", choices=["hero", "reference"])
     ap.add_argument("--workload", default="dit42", choices=["dit42", "aether", "paper_hp", "tiny", "kernels"])
     ap.add_argument("--only", default="", help="kernels workload: comma list of select,extrapolate,gather,scatter,"
-                                               "attention,gemm,block")
+                                               "attention,gemm,deep,block")
     ap.add_argument("--small", action="store_true", help="kernels workload: profiler-sized tensor-core cases")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-collapse", action="store_true", help="skip the deep-stack-collapse variant run")
