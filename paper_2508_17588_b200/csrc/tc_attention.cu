@@ -36,6 +36,9 @@
 #include "hero_internal.h"
 #include "tc_common.cuh"
 
+#ifndef HERO_ATT_CHUNK
+#define HERO_ATT_CHUNK 16
+#endif
 #ifndef HERO_ATT_POLY_OF_8
 #define HERO_ATT_POLY_OF_8 2
 #endif
@@ -64,13 +67,6 @@ static_assert(kKBytes % 1024 == 0 && kKT % 16 == 0, "tile shape");
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-// The same instruction, pinned: the compiler keeps volatile statements in program order, which is how
-// the fused pass below spreads its exponentials evenly through the other arithmetic.
-__device__ __forceinline__ float ex2_pinned(float x) {
-  float y;
-  asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
 __device__ __forceinline__ float max3(float a, float b, float c) {
@@ -159,42 +155,37 @@ __device__ __forceinline__ float softmax_tile(uint32_t t_buf, int valid, float c
 // the row is already scaled by, the tile's own maximum tracked on the side.  The caller checks the
 // maximum afterwards and falls back to softmax_tile (S is still intact: P is only kept in
 // registers here) in the rare case that it has to move.  Doing without the separate maximum pass
-// matters because that pass issues nothing to the exponential unit: two warps of an SM
-// sub-partition then tend to run their exponential phases at the same time and their other
-// phases at the same time, and the unit that bounds the kernel idles in between.  Here every
-// stretch of the instruction stream has the same mix: the exponentials are issued in a fixed
-// order, two pairs behind the multiply that feeds them and three pairs ahead of the code that
-// consumes them, with the scores read 32 columns at a time one chunk ahead.
+// matters because that pass issues nothing to the exponential unit for a third of the tile.  The
+// scores are read kCh columns at a time, one read ahead; short reads keep the register count low
+// enough for the compiler to overlap the pairs freely (16 columns measured 4 % faster than 32).
 __device__ __forceinline__ void fused_tile(uint32_t t_buf, float c, float neg_mc, uint32_t (&packed)[kKT / 2],
                                            float& sum, float& m_tile) {
   const float2 c2 = make_float2(c, c), nm2 = make_float2(neg_mc, neg_mc);
   float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
   float mx[2] = {-INFINITY, -INFINITY};
-  uint32_t ra[32], rb[32];
-  tmem_ld32(t_buf, ra);
+  constexpr int kCh = HERO_ATT_CHUNK;                  // score columns per TMEM read
+  uint32_t ra[kCh], rb[kCh];
+  if (kCh == 32) tmem_ld32(t_buf, *reinterpret_cast<uint32_t(*)[32]>(&ra[0]));
+  else tmem_ld16(t_buf, *reinterpret_cast<uint32_t(*)[16]>(&ra[0]));
 #pragma unroll
-  for (int ch = 0; ch < kKT / 32; ++ch) {
-    uint32_t(&cur)[32] = (ch & 1) ? rb : ra;
-    uint32_t(&nxt)[32] = (ch & 1) ? ra : rb;
+  for (int ch = 0; ch < kKT / kCh; ++ch) {
+    uint32_t(&cur)[kCh] = (ch & 1) ? rb : ra;
+    uint32_t(&nxt)[kCh] = (ch & 1) ? ra : rb;
     tmem_ld_wait();
-    if (ch + 1 < kKT / 32) tmem_ld32(t_buf + (ch + 1) * 32, nxt);
-    float2 x[16], p[16];
-    x[0] = __ffma2_rn(f2(cur[0], cur[1]), c2, nm2);
-    x[1] = __ffma2_rn(f2(cur[2], cur[3]), c2, nm2);
+    if (ch + 1 < kKT / kCh) {
+      if (kCh == 32) tmem_ld32(t_buf + (ch + 1) * kCh, *reinterpret_cast<uint32_t(*)[32]>(&nxt[0]));
+      else tmem_ld16(t_buf + (ch + 1) * kCh, *reinterpret_cast<uint32_t(*)[16]>(&nxt[0]));
+    }
 #pragma unroll
-    for (int i = 0; i < 16 + 3; ++i) {
-      if (i + 2 < 16) x[i + 2] = __ffma2_rn(f2(cur[2 * i + 4], cur[2 * i + 5]), c2, nm2);
-      if (i < 16) {
-        if ((i & 7) < kPolyOf8) p[i] = exp2_poly(x[i]);
-        else { p[i].x = ex2_pinned(x[i].x); p[i].y = ex2_pinned(x[i].y); }
-      }
-      if (i >= 3) {
-        const int k = i - 3;
-        acc[k & 3] = __fadd2_rn(acc[k & 3], p[k]);
-        const __nv_bfloat162 b = __floats2bfloat162_rn(p[k].x, p[k].y);
-        packed[ch * 16 + k] = *reinterpret_cast<const uint32_t*>(&b);
-        mx[k & 1] = max3(mx[k & 1], __uint_as_float(cur[2 * k]), __uint_as_float(cur[2 * k + 1]));
-      }
+    for (int i = 0; i < kCh / 2; ++i) {
+      const float2 x = __ffma2_rn(f2(cur[2 * i], cur[2 * i + 1]), c2, nm2);
+      float2 p;
+      if ((i & 7) < kPolyOf8) p = exp2_poly(x);
+      else { p.x = ex2(x.x); p.y = ex2(x.y); }
+      acc[i & 3] = __fadd2_rn(acc[i & 3], p);
+      const __nv_bfloat162 b = __floats2bfloat162_rn(p.x, p.y);
+      packed[ch * (kCh / 2) + i] = *reinterpret_cast<const uint32_t*>(&b);
+      mx[i & 1] = max3(mx[i & 1], __uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1]));
     }
   }
   const float2 a01 = __fadd2_rn(acc[0], acc[1]), a23 = __fadd2_rn(acc[2], acc[3]);
