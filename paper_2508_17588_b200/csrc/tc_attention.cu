@@ -26,9 +26,10 @@
 //     P V has completed.  The final division by the row sum makes the result independent of
 //     which maximum was used.
 //
-// The exponential unit, not the tensor core, bounds this kernel at head_dim 64 (one ex2 per 256
-// tensor flops): kPolyOf8 of every 8 score pairs take 2^x from a degree-3 polynomial on the FMA
-// pipe instead (Cody-Waite split x = n + f, |f| <= 1/2, exponent bits added as an integer).
+// At head_dim 64 the softmax, not the tensor core, bounds this kernel: one ex2 (16 per clock per SM),
+// one bf16 conversion, one running-maximum and one row-sum update per score against 256 tensor flops.
+// Evaluating part of the exponentials with a polynomial on the FMA pipe was measured and brings
+// nothing: the per-score instruction mix runs at 16-17 cycles per warp-pair of scores either way.
 #include <cuda.h>
 
 #include <mutex>
@@ -38,9 +39,6 @@
 
 #ifndef HERO_ATT_CHUNK
 #define HERO_ATT_CHUNK 16
-#endif
-#ifndef HERO_ATT_POLY_OF_8
-#define HERO_ATT_POLY_OF_8 2
 #endif
 
 namespace hero {
@@ -59,7 +57,6 @@ constexpr int kFirstSoftmaxWarp = 4;
 constexpr int kAttThreads = 32 * (kFirstSoftmaxWarp + 4 * kQTiles);   // 12 warps
 constexpr size_t kAttSmem = 1024 + kQTiles * kQBytes + (size_t)kKvStages * kKvStageBytes + 512;
 constexpr uint32_t kTileCols = 256, kColO = 2 * kKT, kAttTmemCols = 512;   // per tile: S0 | S1 | O
-constexpr int kPolyOf8 = HERO_ATT_POLY_OF_8;   // score pairs per 8 whose 2^x comes from the polynomial
 constexpr float kRescaleLog2 = 8.0f;           // the scaling maximum moves only when exceeded by 2^8
 static_assert(2 * kKT + kHD <= (int)kTileCols && kQTiles * kTileCols <= kAttTmemCols, "TMEM layout");
 static_assert(kKBytes % 1024 == 0 && kKT % 16 == 0, "tile shape");
@@ -75,25 +72,6 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   return y;
 }
 __device__ __forceinline__ float2 f2(uint32_t a, uint32_t b) { return make_float2(__uint_as_float(a), __uint_as_float(b)); }
-
-// 2^x for a pair, x <= 8, on the FMA and integer pipes.  x is clamped at -126 so that the
-// exponent arithmetic stays inside the normal range; t = x + 1.5*2^23 holds round(x) in its low
-// mantissa bits, f = x - round(x) lies in [-1/2, 1/2], the cubic (minimax in relative error,
-// 7.5e-5, far below the bf16 rounding of P) gives 2^f, and round(x) is added to the exponent field.
-__device__ __forceinline__ float2 exp2_poly(float2 x) {
-  const float kMagic = 12582912.0f;
-  x.x = fmaxf(x.x, -126.0f);
-  x.y = fmaxf(x.y, -126.0f);
-  const float2 t = __fadd2_rn(x, make_float2(kMagic, kMagic));
-  const float2 n = __fadd2_rn(t, make_float2(-kMagic, -kMagic));
-  const float2 f = __ffma2_rn(n, make_float2(-1.0f, -1.0f), x);
-  float2 p = __ffma2_rn(f, make_float2(0.0551716648042202f, 0.0551716648042202f),
-                        make_float2(0.2426111251115799f, 0.2426111251115799f));
-  p = __ffma2_rn(p, f, make_float2(0.6932609677314758f, 0.6932609677314758f));
-  p = __ffma2_rn(p, f, make_float2(0.9999280571937561f, 0.9999280571937561f));
-  return make_float2(__uint_as_float(__float_as_uint(p.x) + (__float_as_uint(t.x) << 23)),
-                     __uint_as_float(__float_as_uint(p.y) + (__float_as_uint(t.y) << 23)));
-}
 
 // One key tile of one query row.  The kKT scores of the row are read from TMEM in one burst
 // (a single wait for the whole row instead of one per chunk), reduced to their maximum, turned
@@ -134,9 +112,7 @@ __device__ __forceinline__ float softmax_tile(uint32_t t_buf, int valid, float c
     for (int i = 0; i < 16; ++i) {       // pair i = columns 2i, 2i+1 of this 32-column chunk
       const int col = ch * 32 + 2 * i;
       const float2 x = __ffma2_rn(f2(s[col], s[col + 1]), c2, nm2);
-      float2 p;
-      if (!MASKED && (i & 7) < kPolyOf8) p = exp2_poly(x);
-      else p = make_float2(ex2(x.x), ex2(x.y));
+      float2 p = make_float2(ex2(x.x), ex2(x.y));
       if (MASKED) {
         if (col >= valid) p.x = 0.f;
         if (col + 1 >= valid) p.y = 0.f;
@@ -179,9 +155,7 @@ __device__ __forceinline__ void fused_tile(uint32_t t_buf, float c, float neg_mc
 #pragma unroll
     for (int i = 0; i < kCh / 2; ++i) {
       const float2 x = __ffma2_rn(f2(cur[2 * i], cur[2 * i + 1]), c2, nm2);
-      float2 p;
-      if ((i & 7) < kPolyOf8) p = exp2_poly(x);
-      else { p.x = ex2(x.x); p.y = ex2(x.y); }
+      const float2 p = make_float2(ex2(x.x), ex2(x.y));
       acc[i & 3] = __fadd2_rn(acc[i & 3], p);
       const __nv_bfloat162 b = __floats2bfloat162_rn(p.x, p.y);
       packed[ch * (kCh / 2) + i] = *reinterpret_cast<const uint32_t*>(&b);
