@@ -33,7 +33,7 @@ sys.path.insert(0, ROOT)
 from workloads import synthetic as S  # noqa: E402
 
 METRIC = "hero_cached_step_tokens_per_s"
-ATTENTION_TRAFFIC_RATIO = 1.003   # dram__bytes_read+write / algorithmic bytes of tc_attention_kernel (ncu, small case)
+ATTENTION_TRAFFIC_RATIO = 1.002   # dram__bytes_read+write / algorithmic bytes of tc_attention_kernel (ncu, small case)
 UNIT = "tokens/s"
 
 
@@ -309,7 +309,7 @@ def run_hero(args, cfg, rank, world, local_rank):
         gemm_ms_blk = prof["gemm"][0] / prof["attention"][1]          # four GEMMs per attention launch
         achieved = fl["attention"] / (att_ms * 1e-3) / 1e12
         peak = peaks["bf16_tflops_sustained"]
-        # DRAM bytes per launch: an ncu capture of a smaller launch of this kernel read and wrote 1.003 x its
+        # DRAM bytes per launch: an ncu capture of a smaller launch of this kernel read and wrote 1.002 x its
         # algorithmic bytes (K and V once, Q in, O out); the traffic grows in proportion with those, so the
         # full launch is that ratio times its own algorithmic bytes
         alg_bytes = 2 * B * N * D * 2 + 2 * B * n_sel * D * 2
