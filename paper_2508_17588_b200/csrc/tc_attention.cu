@@ -10,9 +10,8 @@
 //                 N-contiguous shared-memory operand.  Each tile has its own issuer so that
 //                 neither tile's hand-shakes can hold up the other's.
 //   warps 4..7    softmax group of query tile 0, warps 8..11 of query tile 1: one thread per
-//                 query row, which holds the row's 96 scores of a key tile in registers (one TMEM
-//                 read burst per tile); running max / sum in registers, P written back over S
-//                 in TMEM as bf16
+//                 query row; running max / sum in registers, the scores of a key tile read from
+//                 TMEM 16 columns at a time, P written back over S in TMEM as bf16
 // TMEM (512 columns): per query tile two S buffers of 96 columns (key tile parity) and one
 // 64-column output accumulator; P (48 columns of bf16 pairs) overwrites the head of its S buffer.
 //

@@ -90,6 +90,34 @@ def test_attention_peaked_rows():
     assert np.abs(to_host(o)[0] - v[0, pick]).max() <= 2e-2
 
 
+@pytest.mark.parametrize("N", [960, 1000, 97, 193])
+def test_attention_scores_that_keep_growing(N):
+    """Keys whose scores grow steadily along the sequence: the running maximum has to move again and again
+    (by more than the 2^8 slack), so the accumulator is rescaled in many key tiles, on both tile parities,
+    including the ragged last tile; rows with a flat score profile sit in the same warps."""
+    rng = np.random.default_rng(N)
+    n_q, D = 200, 64
+    base = rng.standard_normal(D).astype(np.float32)
+    base /= np.linalg.norm(base)
+    ramp = np.linspace(0.0, 60.0, N, dtype=np.float32)[:, None]                    # score ~ 8 * ramp * |q.base|
+    k = S.round_bf16((rng.standard_normal((1, N, D)) * 0.3 + ramp * base).astype(np.float32))
+    v = S.round_bf16(rng.standard_normal((1, N, D)).astype(np.float32))
+    q = rng.standard_normal((1, n_q, D)).astype(np.float32) * 0.3
+    q[:, ::2] += 8.0 * base                                                        # every other row climbs the ramp
+    q[:, 1::4] -= 8.0 * base                                                       # some descend it
+    q = S.round_bf16(q)
+    cfg = O.Config(n_blocks=1, n_shallow=1, hidden=D, n_heads=1, head_dim=64, ffn_dim=8, temb_dim=8, batch=1,
+                   frames=1, grid_h=1, grid_w=1, n_text=0, patch_h=1, patch_w=1, ratio_num=1, ratio_den=1)
+    o = torch.full((1, n_q, D), float("nan"), device="cuda", dtype=torch.bfloat16)
+    H().hero_attention_bf16(to_dev(q, "bf16"), to_dev(k, "bf16"), to_dev(v, "bf16"), o, 1)
+    H().hero_isolated_status()
+    got = to_host(o)[0]
+    assert np.isfinite(got).all()
+    want = O.attention(cfg, q[0].astype(np.float64), k[0].astype(np.float64), v[0].astype(np.float64))
+    assert rel_l2(got, want) <= 1e-2
+    assert np.abs(got - want).max() <= 3e-2 * np.abs(want).max()
+
+
 # ---------------------------------------------------------------- bf16 blocks
 SMALL_BF16 = dict(n_blocks=2, n_shallow=1, hidden=256, n_heads=4, head_dim=64, ffn_dim=768, temb_dim=64, batch=2,
                   frames=3, grid_h=9, grid_w=11, n_text=10, patch_h=2, patch_w=2, ratio_num=1, ratio_den=4,
