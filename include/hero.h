@@ -62,6 +62,11 @@ typedef struct hero_config {
   int has_gate;            /* 1: adaLN also yields a gate per branch (6 chunks instead of 4) */
   unsigned long long seed; /* low 32 bits seed the sampler's counter-based hash */
   int deep_collapse;       /* 1: hero_step keeps ONE history pair for the whole deep stack (see below) */
+  int track_mode;          /* frequency-aware tracking (Sec. 4.3): 0 = weighted draw, key (age+1)*(hash+1);
+                              1 = strict oldest-first, key (age, hash): the longest-unsampled tokens of a
+                              patch always win, the hash only breaks ties */
+  int share_selection;     /* 1: hero_step draws ONE list per cached step (block 0's sampler and age
+                              counters) and every shallow block refreshes those rows */
 } hero_config;
 
 /* Device pointers to one block's parameters (borrowed for the context's lifetime).

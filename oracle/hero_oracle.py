@@ -61,6 +61,8 @@ class Config:
     warmup_full_steps: int = 2
     full_interval: int = 0    # M; 0 = never again after warm-up
     has_gate: int = 0
+    track_mode: int = 0       # 0: weighted draw (age+1)*(hash+1); 1: strict oldest-first (age, hash)
+    share_selection: int = 0  # 1: one list per cached step (block 0's sampler) for every shallow block
     seed: int = 0
     eps: float = 1e-5
 
@@ -162,8 +164,10 @@ def select_tokens(cfg: Config, ages: np.ndarray, block: int, call: int):
 
     Each token draws U = (h+1) with h a 32-bit hash and competes with key
     (age+1) * U: a uniform draw on (0, age+1] up to scale, so the chance of being
-    picked grows with age and is uniform when ages are equal.  The q_i largest keys
-    of patch i win (ties: lower token index first).  Ages: picked -> 0, others +1
+    picked grows with age and is uniform when ages are equal (track_mode 0); with
+    track_mode 1 the key is (age, hash): the longest-unsampled tokens always win and the
+    draw only orders tokens of equal age.  The q_i largest keys of patch i win (ties:
+    lower token index first).  Ages: picked -> 0, others +1
     (saturating).  Returns (sequence rows ascending, new ages)."""
     ages = np.asarray(ages)
     assert ages.shape == (cfg.n_video,)
@@ -171,7 +175,11 @@ def select_tokens(cfg: Config, ages: np.ndarray, block: int, call: int):
     for toks, q in zip(patch_table(cfg), patch_quotas(cfg, call)):
         keyed = []
         for v in toks:
-            key = (int(ages[v]) + 1) * (token_hash(cfg.seed, block, call, v) + 1)
+            h = token_hash(cfg.seed, block, call, v)
+            if cfg.track_mode == 0:
+                key = (int(ages[v]) + 1) * (h + 1)
+            else:                                   # strict oldest-first: the draw only orders equal ages
+                key = (int(ages[v]) << 32) | h
             keyed.append((-key, v))
         for _, v in sorted(keyed)[:q]:
             picked[v] = True
@@ -376,9 +384,10 @@ class HeroOracle:
         s_last = self.full_steps[-1]
         d = s_last - self.full_steps[-2] if len(self.full_steps) > 1 else 1
         k = s - s_last
+        shared = self.select(0) if (c.share_selection and c.n_shallow > 0) else None
         for l in range(c.n_blocks):
             if l < c.n_shallow:
-                rows = self.select(l)
+                rows = shared if shared is not None else self.select(l)
                 self.block_refresh(l, x, temb, rows)
             else:
                 self.block_extrapolate(l, x, k, d)

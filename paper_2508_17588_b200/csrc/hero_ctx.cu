@@ -106,7 +106,7 @@ SelectGeom geom_of(const hero_config& c) {
   SelectGeom g;
   g.frames = c.frames; g.grid_h = c.grid_h; g.grid_w = c.grid_w; g.n_text = c.n_text;
   g.patch_h = c.patch_h; g.patch_w = c.patch_w;
-  g.ratio_num = c.ratio_num; g.ratio_den = c.ratio_den; g.quota_mode = c.quota_mode;
+  g.ratio_num = c.ratio_num; g.ratio_den = c.ratio_den; g.quota_mode = c.quota_mode; g.track_mode = c.track_mode;
   g.seed_lo = (uint32_t)(c.seed & 0xFFFFFFFFull);
   return g;
 }
@@ -268,6 +268,8 @@ int validate(const hero_config* g) {
   if (g->dtype != HERO_DTYPE_FP32 && g->dtype != HERO_DTYPE_BF16) return HERO_ERR_ARG;
   if (g->n_shallow > kMaxSelectBatch) return HERO_ERR_ARG;
   if (g->deep_collapse != 0 && g->deep_collapse != 1) return HERO_ERR_ARG;
+  if (g->track_mode != 0 && g->track_mode != 1) return HERO_ERR_ARG;
+  if (g->share_selection != 0 && g->share_selection != 1) return HERO_ERR_ARG;
   if (g->dtype == HERO_DTYPE_BF16) {
     if (g->head_dim != 64 || g->hidden % 8 || g->ffn_dim % 8 || g->temb_dim % 8) return HERO_ERR_ALIGN;
   } else {
@@ -511,10 +513,12 @@ int hero_step(hero_ctx* c, int step, void* d_x, const void* d_temb) {
   if (k <= 0 || d <= 0) return HERO_ERR_STATE;
   // all shallow blocks draw their lists in one launch: the draw depends on counters only
   int n_sel[kMaxSelectBatch];
+  // one list for the whole step (drawn with block 0's sampler) or one per shallow block
+  const int n_draws = g.share_selection ? (g.n_shallow > 0 ? 1 : 0) : g.n_shallow;
   if (g.n_shallow > 0) {
     SelectBatch batch;
-    batch.n = g.n_shallow;
-    for (int l = 0; l < g.n_shallow; ++l) {
+    batch.n = n_draws;
+    for (int l = 0; l < n_draws; ++l) {
       BlockMem& bm = c->blk[l];
       n_sel[l] = n_sel_for_call(c, bm.calls);
       batch.block[l] = l; batch.call[l] = bm.calls;
@@ -522,12 +526,13 @@ int hero_step(hero_ctx* c, int step, void* d_x, const void* d_temb) {
       batch.idx[l] = c->idx_ws + (size_t)l * c->idx_cap;
     }
     HERO_LAUNCH(c, HERO_PROF_SELECT, launch_select(geom_of(g), batch, c->stream));
-    for (int l = 0; l < g.n_shallow; ++l) { c->blk[l].ages_cur ^= 1; c->blk[l].calls++; }
+    for (int l = 0; l < n_draws; ++l) { c->blk[l].ages_cur ^= 1; c->blk[l].calls++; }
+    for (int l = n_draws; l < g.n_shallow; ++l) n_sel[l] = n_sel[0];
   }
   for (int l = 0; l < g.n_blocks; ++l) {
     if (l < g.n_shallow) {
       if (n_sel[l] > 0) {
-        HERO_TRY(refresh_block(c, l, d_x, d_temb, c->idx_ws + (size_t)l * c->idx_cap, n_sel[l]));
+        HERO_TRY(refresh_block(c, l, d_x, d_temb, c->idx_ws + (size_t)(g.share_selection ? 0 : l) * c->idx_cap, n_sel[l]));
       } else {
         HERO_LAUNCH(c, HERO_PROF_RESIDUAL,
                     launch_residual2(d_x, c->blk[l].g[0], c->blk[l].g[1], c->elems, g.dtype, c->stream));

@@ -55,7 +55,7 @@ struct GemmOut {
 struct SelectGeom {
   int frames, grid_h, grid_w, n_text;
   int patch_h, patch_w;
-  int ratio_num, ratio_den, quota_mode;
+  int ratio_num, ratio_den, quota_mode, track_mode;
   uint32_t seed_lo;
 };
 constexpr int kMaxSelectBatch = 64;

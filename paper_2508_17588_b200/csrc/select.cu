@@ -23,6 +23,14 @@ __device__ __forceinline__ uint32_t mix32(uint32_t x) {
   return x;
 }
 
+// Sampling key of a token: larger wins.  Mode 0: (age+1) * (hash+1), a uniform draw on (0, age+1] up to
+// scale, so the chance of being picked grows with the time a token has gone unsampled.  Mode 1: age first,
+// hash second - strict oldest-first, the draw only orders tokens of equal age.
+__device__ __forceinline__ unsigned long long make_key(int track_mode, uint32_t age, uint32_t hash) {
+  return track_mode == 0 ? (unsigned long long)(age + 1u) * ((unsigned long long)hash + 1ull)
+                         : ((unsigned long long)age << 32) | (unsigned long long)hash;
+}
+
 __global__ void __launch_bounds__(kSelThreads) select_kernel(const SelectGeom g, const SelectBatch batch) {
   const int e = blockIdx.x;
   if (e >= batch.n) return;
@@ -65,15 +73,13 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const SelectGeom g,
         quota = min(n_here, (int)((2ll * n_here * ra + rb) / (2 * rb)));
       }
       age_v = ages_in[v];
-      const unsigned long long key_v =
-          (unsigned long long)(age_v + 1u) * ((unsigned long long)mix32(h_block + (uint32_t)v) + 1ull);
+      const unsigned long long key_v = make_key(g.track_mode, age_v, mix32(h_block + (uint32_t)v));
       int beaten_by = 0;
       for (int dy = 0; dy < hh; ++dy) {
         for (int dx = 0; dx < ww; ++dx) {
           const int u = (t * H + y0 + dy) * W + x0 + dx;
           if (u == v) continue;
-          const unsigned long long key_u = (unsigned long long)((uint32_t)ages_in[u] + 1u) *
-                                           ((unsigned long long)mix32(h_block + (uint32_t)u) + 1ull);
+          const unsigned long long key_u = make_key(g.track_mode, (uint32_t)ages_in[u], mix32(h_block + (uint32_t)u));
           beaten_by += (key_u > key_v || (key_u == key_v && u < v)) ? 1 : 0;
         }
       }

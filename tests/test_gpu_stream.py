@@ -120,6 +120,8 @@ SEL_CASES = {
     "cogvideo_25": dict(S.CONFIGS["kernels"], dtype="fp32", hidden=64, n_heads=1, ffn_dim=64, temb_dim=8),
     "aether_10": dict(S.CONFIGS["aether"], dtype="fp32", hidden=64, n_heads=1, ffn_dim=64, temb_dim=8,
                       n_blocks=2, n_shallow=2, ratio_num=1, ratio_den=10),
+    "oldest_first": dict(S.CONFIGS["tiny"], frames=3, grid_h=7, grid_w=9, patch_h=2, patch_w=3, ratio_num=1,
+                         ratio_den=3, track_mode=1, seed=4),
     "paper_2x3_r02": dict(S.CONFIGS["kernels"], dtype="fp32", hidden=64, n_heads=1, ffn_dim=64, temb_dim=8,
                           frames=11, patch_h=2, patch_w=3, ratio_num=1, ratio_den=5, quota_mode=1),
 }

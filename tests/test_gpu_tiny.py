@@ -173,3 +173,24 @@ def test_paper_hyperparameters_small_model():
             assert int(hero.hero_state_get(l, "calls")[0]) == orc.blocks[l].calls
     assert n_full == 5
     hero.close()
+
+
+@pytest.mark.parametrize("variant", [dict(track_mode=1), dict(share_selection=1), dict(track_mode=1, share_selection=1, deep_collapse=1)])
+def test_tracking_and_selection_variants(variant):
+    """Strict oldest-first tracking, one selection list shared by all refresh blocks of a step, and both
+    together with the collapsed deep stack: 8 steps through hero_step against the oracle."""
+    cfgd = dict(S.CONFIGS["tiny"], n_blocks=5, n_shallow=3, full_interval=3, steps=8, seed=21, **variant)
+    orc, hero, _ = make_pair(cfgd)
+    x_host = S.tokens(cfgd)
+    for s in range(cfgd["steps"]):
+        temb = S.temb(cfgd, s)
+        want = orc.step(s, x_host, temb)
+        x = to_dev(x_host, "fp32")
+        hero.hero_step(s, x, to_dev(temb, "fp32"))
+        assert rel_l2(to_host(x), want) <= FP32_TOL, s
+        for l in range(cfgd["n_shallow"]):
+            assert np.array_equal(hero.hero_state_get(l, "ages").numpy(), orc.blocks[l].ages), (s, l)
+            assert int(hero.hero_state_get(l, "calls")[0]) == orc.blocks[l].calls
+    if variant.get("share_selection"):
+        assert orc.blocks[1].calls == 0 and orc.blocks[0].calls > 0       # only block 0's sampler is used
+    hero.close()

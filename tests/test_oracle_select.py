@@ -9,6 +9,7 @@ import numpy as np
 import pytest
 
 from oracle import hero_oracle as O
+from workloads import synthetic as S
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
@@ -250,3 +251,45 @@ def test_draws_differ_between_blocks_and_calls():
     assert not np.array_equal(a, b) and not np.array_equal(a, c)
     a2, _ = O.select_tokens(cfg, z, 0, 0)
     assert np.array_equal(a, a2)
+
+
+# ---------------------------------------------------------------- strict oldest-first tracking (track_mode 1)
+def test_oldest_first_never_leaves_a_token_unsampled_longer_than_one_round():
+    """With the key (age, hash) a patch of #P tokens and quota q samples every token once per
+    ceil(#P / q) calls: ages never exceed that bound (the guarantee the tracking paragraph asks for)."""
+    cfgd = dict(S.CONFIGS["tiny"], frames=2, grid_h=6, grid_w=6, patch_h=2, patch_w=3, ratio_num=1, ratio_den=3,
+                quota_mode=1, track_mode=1, seed=3)
+    cfg = O.Config.from_dict(cfgd)
+    assert set(O.patch_quotas(cfg, 0)) == {2}                      # 6-token patches, two per call
+    ages = np.zeros(cfg.n_video, np.uint16)
+    seen = np.zeros(cfg.n_video, int)
+    for call in range(12):
+        rows, ages = O.select_tokens(cfg, ages, 0, call)
+        seen[rows - cfg.n_text] += 1
+        assert ages.max() <= 2                                     # ceil(6/2) - 1
+        if (call + 1) % 3 == 0:
+            assert (seen == (call + 1) // 3).all()                 # exact round robin, order decided by the hash
+    # the weighted mode has no such bound: some token waits longer over the same calls
+    cfg0 = O.Config.from_dict(dict(cfgd, track_mode=0))
+    ages, worst = np.zeros(cfg0.n_video, np.uint16), 0
+    for call in range(12):
+        _, ages = O.select_tokens(cfg0, ages, 0, call)
+        worst = max(worst, int(ages.max()))
+    assert worst > 2
+
+
+def test_oldest_first_prefers_age_over_any_draw_and_uses_the_draw_among_equals():
+    cfgd = dict(S.CONFIGS["tiny"], frames=1, grid_h=2, grid_w=2, patch_h=2, patch_w=2, ratio_num=1, ratio_den=4,
+                track_mode=1, n_text=0)
+    cfg = O.Config.from_dict(cfgd)
+    for seed in range(40):
+        c = O.Config.from_dict(dict(cfgd, seed=seed))
+        ages = np.array([0, 3, 1, 2], np.uint16)
+        rows, new = O.select_tokens(c, ages, 0, 0)
+        assert list(rows) == [1]                                   # the oldest token, whatever the draw
+        assert list(new) == [1, 0, 2, 3]
+    winners = set()
+    for seed in range(40):                                         # equal ages: the draw decides
+        rows, _ = O.select_tokens(O.Config.from_dict(dict(cfgd, seed=seed)), np.zeros(4, np.uint16), 0, 0)
+        winners.add(int(rows[0]))
+    assert winners == {0, 1, 2, 3}
