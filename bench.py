@@ -346,29 +346,38 @@ def run_hero(args, cfg, rank, world, local_rank):
     mem = hero.hero_device_bytes()
     hero.close()
 
-    # the same cached step with the deep stack collapsed to one history pair (a variant: not the headline)
-    collapsed = None
-    if cfg["n_shallow"] < cfg["n_blocks"] and not args.no_collapse:
-        hero = H.Hero(dict(run_cfg, deep_collapse=1), weights)
+    # the same cached step under two opt-in variants (reported beside the headline, never as it)
+    def time_variant(extra):
+        hv = H.Hero(dict(run_cfg, **extra), weights)
         for s_ in range(2):
-            hero.hero_step(s_, x, tembs[s_])
+            hv.hero_step(s_, x, tembs[s_])
         st = 2
         for _ in range(args.warmup):
-            hero.hero_step(st, x, tembs[st % 8]); st += 1
+            hv.hero_step(st, x, tembs[st % 8]); st += 1
         n_c = max(2, min(args.steps, 5))
         torch.cuda.synchronize()
         e0, e1 = ev(), ev()
         e0.record()
         for _ in range(n_c):
-            hero.hero_step(st, x, tembs[st % 8]); st += 1
+            hv.hero_step(st, x, tembs[st % 8]); st += 1
         e1.record()
         torch.cuda.synchronize()
-        hero.hero_check_status()
-        c_ms = max_over_ranks(e0.elapsed_time(e1) / n_c, dist, device)
-        collapsed = {"ms_per_step": c_ms, "value": whole_job_throughput(tokens, world, c_ms), "unit": UNIT,
-                     "device_bytes": hero.hero_device_bytes(),
-                     "note": "deep_collapse=1: Eq. 5 applied once to the fp32 sum of the deep blocks' branch outputs"}
-        hero.close()
+        hv.hero_check_status()
+        v_ms = max_over_ranks(e0.elapsed_time(e1) / n_c, dist, device)
+        out = {"ms_per_step": v_ms, "value": whole_job_throughput(tokens, world, v_ms), "unit": UNIT,
+               "device_bytes": hv.hero_device_bytes()}
+        hv.close()
+        return out
+
+    collapsed = attend_refreshed = None
+    if not args.no_collapse:
+        if cfg["n_shallow"] < cfg["n_blocks"]:
+            collapsed = time_variant(dict(deep_collapse=1))
+            collapsed["note"] = "deep_collapse=1: Eq. 5 applied once to the fp32 sum of the deep blocks' branch outputs"
+        if cfg["n_shallow"] > 0:
+            attend_refreshed = time_variant(dict(attend_mode=1))
+            attend_refreshed["note"] = ("attend_mode=1: the refreshed queries of a cached step attend to the refreshed "
+                                        "and text rows only (Eq. 3 read literally) instead of the full cached K/V")
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -398,6 +407,8 @@ def run_hero(args, cfg, rank, world, local_rank):
                 "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "breakdown_ms": breakdown}
         if collapsed:
             line["deep_collapse_variant"] = collapsed
+        if attend_refreshed:
+            line["attend_refreshed_variant"] = attend_refreshed
         if roofline:
             line["roofline"] = roofline
         if cpu_baseline:
@@ -571,7 +582,7 @@ def main():
                                                "attention,gemm,deep,block")
     ap.add_argument("--small", action="store_true", help="kernels workload: profiler-sized tensor-core cases")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-collapse", action="store_true", help="skip the deep-stack-collapse variant run")
+    ap.add_argument("--no-collapse", action="store_true", help="skip the variant runs (collapsed deep stack, refreshed-rows-only attention)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

@@ -67,6 +67,9 @@ typedef struct hero_config {
                               patch always win, the hash only breaks ties */
   int share_selection;     /* 1: hero_step draws ONE list per cached step (block 0's sampler and age
                               counters) and every shallow block refreshes those rows */
+  int attend_mode;         /* which keys the refreshed queries of a cached step attend to: 0 = the full cached
+                              K/V of all rows (default); 1 = only the rows refreshed in this step plus the
+                              text rows (Eq. 3 read literally, F(S(z), S(tau)) with the text kept) */
 } hero_config;
 
 /* Device pointers to one block's parameters (borrowed for the context's lifetime).

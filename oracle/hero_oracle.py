@@ -63,6 +63,7 @@ class Config:
     has_gate: int = 0
     track_mode: int = 0       # 0: weighted draw (age+1)*(hash+1); 1: strict oldest-first (age, hash)
     share_selection: int = 0  # 1: one list per cached step (block 0's sampler) for every shallow block
+    attend_mode: int = 0      # 0: refreshed queries see the full cached K/V; 1: refreshed + text rows only
     seed: int = 0
     eps: float = 1e-5
 
@@ -325,7 +326,12 @@ class HeroOracle:
             st.k_cache[b, rows] = k
             st.v_cache[b, rows] = v
             sel = np.searchsorted(rows, rows_out)
-            o = attention(c, q[sel], st.k_cache[b], st.v_cache[b])
+            if c.attend_mode == 1 and not full:
+                # Eq. 3 read literally, F(S(z), S(tau)), with the (never refreshed) text rows kept
+                seen = np.concatenate([np.arange(c.n_text), rows])
+                o = attention(c, q[sel], st.k_cache[b][seen], st.v_cache[b][seen])
+            else:
+                o = attention(c, q[sel], st.k_cache[b], st.v_cache[b])
             g = o @ w["w_o"].T + w["b_o"]
             if c.has_gate:
                 g = g * gate1[b]

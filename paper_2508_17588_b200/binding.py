@@ -35,7 +35,7 @@ class HeroConfig(C.Structure):
         "n_blocks", "n_shallow", "hidden", "n_heads", "head_dim", "ffn_dim", "temb_dim",
         "batch", "frames", "grid_h", "grid_w", "n_text", "patch_h", "patch_w",
         "ratio_num", "ratio_den", "quota_mode", "warmup_full_steps", "full_interval", "dtype", "has_gate")
-    ] + [("seed", C.c_ulonglong), ("deep_collapse", C.c_int), ("track_mode", C.c_int), ("share_selection", C.c_int)]
+    ] + [("seed", C.c_ulonglong), ("deep_collapse", C.c_int), ("track_mode", C.c_int), ("share_selection", C.c_int), ("attend_mode", C.c_int)]
 
 
 class HeroBlockWeights(C.Structure):

@@ -46,6 +46,9 @@ struct hero_ctx {
   void* deep_g[2] = {nullptr, nullptr};
   float* stack_hist[2] = {nullptr, nullptr};
   int stack_last = 0, stack_n = 0, stack_new = 0;
+  // attend_mode 1: compact K/V of the rows a cached step attends to (text + refreshed) and their list
+  void* kv_cmp[2] = {nullptr, nullptr};
+  int* att_list = nullptr;
   void *ws_a = nullptr, *ws_q = nullptr, *ws_o = nullptr, *ws_u = nullptr;
   float* mod = nullptr;                  // [B, n_mod*D] adaLN vectors of the current block
   int* idx_ws = nullptr;                 // [n_shallow, idx_cap] selection lists of the current step
@@ -197,7 +200,24 @@ int refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, const i
   o_qkv.ptr[2] = vdst;    o_qkv.ld[2] = D; o_qkv.scatter[2] = 1;
   o_qkv.seg_cols = D; o_qkv.idx = d_idx; o_qkv.n_sel = n_sel; o_qkv.n_rows = N;
   HERO_TRY(run_gemm(c, c->ws_a, w.w_qkv, w.b_qkv, M, 3 * D, D, o_qkv));
-  HERO_TRY(run_attention(c, c->ws_q, kdst, vdst, c->ws_o, n_sel));
+  if (g.attend_mode == 1 && !full) {
+    // Eq. 3 read literally: the refreshed queries see the refreshed rows (just written) and the text rows
+    const int n_att = g.n_text + n_sel;
+    HERO_LAUNCH(c, HERO_PROF_GATHER_LN, launch_attend_list(d_idx, n_sel, g.n_text, c->att_list, c->stream));
+    HERO_LAUNCH(c, HERO_PROF_GATHER_LN,
+                launch_gather_rows(kdst, c->att_list, c->kv_cmp[0], B, N, n_att, D, g.dtype, c->stream));
+    HERO_LAUNCH(c, HERO_PROF_GATHER_LN,
+                launch_gather_rows(vdst, c->att_list, c->kv_cmp[1], B, N, n_att, D, g.dtype, c->stream));
+    LaunchScope scope(c, HERO_PROF_ATTENTION);
+    if (g.dtype == HERO_DTYPE_BF16)
+      HERO_TRY(launch_tc_attention(c->ws_q, c->kv_cmp[0], c->kv_cmp[1], c->ws_o, B, n_sel, n_att, g.n_heads, c->d_status,
+                                   c->stream));
+    else
+      HERO_TRY(launch_simt_attention(c->ws_q, c->kv_cmp[0], c->kv_cmp[1], c->ws_o, B, n_sel, n_att, g.n_heads, g.head_dim,
+                                     g.dtype, c->stream));
+  } else {
+    HERO_TRY(run_attention(c, c->ws_q, kdst, vdst, c->ws_o, n_sel));
+  }
   GemmOut o_attn = {};
   o_attn.ptr[0] = ga; o_attn.ld[0] = D; o_attn.scatter[0] = 1;
   o_attn.seg_cols = D; o_attn.idx = d_idx; o_attn.n_sel = n_sel; o_attn.n_rows = N;
@@ -270,6 +290,7 @@ int validate(const hero_config* g) {
   if (g->deep_collapse != 0 && g->deep_collapse != 1) return HERO_ERR_ARG;
   if (g->track_mode != 0 && g->track_mode != 1) return HERO_ERR_ARG;
   if (g->share_selection != 0 && g->share_selection != 1) return HERO_ERR_ARG;
+  if (g->attend_mode != 0 && g->attend_mode != 1) return HERO_ERR_ARG;
   if (g->dtype == HERO_DTYPE_BF16) {
     if (g->head_dim != 64 || g->hidden % 8 || g->ffn_dim % 8 || g->temb_dim % 8) return HERO_ERR_ALIGN;
   } else {
@@ -354,6 +375,10 @@ int hero_init(hero_ctx** out, const hero_config* cfg, const hero_block_weights* 
     A((void**)&c->stack_hist[1], (size_t)c->elems * sizeof(float));
   }
   if (cfg->n_shallow < cfg->n_blocks) { A(&c->kv_tmp[0], tensor); A(&c->kv_tmp[1], tensor); }
+  if (cfg->attend_mode == 1) {
+    A(&c->kv_cmp[0], tensor); A(&c->kv_cmp[1], tensor);
+    A((void**)&c->att_list, (size_t)c->N * sizeof(int));
+  }
   A(&c->ws_a, tensor); A(&c->ws_q, tensor); A(&c->ws_o, tensor);
   A(&c->ws_u, (size_t)cfg->batch * c->N * cfg->ffn_dim * c->esz);
   A((void**)&c->mod, (size_t)cfg->batch * c->n_mod * cfg->hidden * sizeof(float));

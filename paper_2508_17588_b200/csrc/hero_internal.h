@@ -84,6 +84,8 @@ int launch_residual2(void* x, const void* ga, const void* gf, long long n, int d
 int launch_residual2_acc(void* x, const void* ga, const void* gf, float* acc, long long n, int dtype, cudaStream_t s);
 int launch_extrapolate_stack(void* x, const float* s_prev, const float* s_last, long long n, int k, int d, int dtype,
                              cudaStream_t s);
+// list[i] = i for i < n_text, list[n_text + i] = idx[i] for i < n_sel (rows a literal Eq. 3 attends to)
+int launch_attend_list(const int* idx, int n_sel, int n_text, int* list, cudaStream_t s);
 int launch_gather_rows(const void* src, const int* idx, void* dst, int B, int N, int n_sel, int D,
                        int dtype, cudaStream_t s);
 int launch_scatter_rows(const void* src, const int* idx, void* dst, int B, int N, int n_sel, int D,

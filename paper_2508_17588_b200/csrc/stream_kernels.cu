@@ -589,6 +589,18 @@ int launch_extrapolate_stack(void* x, const float* s_prev, const float* s_last, 
   return HERO_OK;
 }
 
+static __global__ void attend_list_kernel(const int* __restrict__ idx, int n_sel, int n_text, int* __restrict__ list) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n_text) list[i] = i;
+  else if (i < n_text + n_sel) list[i] = idx[i - n_text];
+}
+int launch_attend_list(const int* idx, int n_sel, int n_text, int* list, cudaStream_t s) {
+  const int n = n_text + n_sel;
+  if (n <= 0) return HERO_OK;
+  attend_list_kernel<<<(n + 255) / 256, 256, 0, s>>>(idx, n_sel, n_text, list);
+  HERO_CUDA_TRY(cudaGetLastError());
+  return HERO_OK;
+}
 static int move_rows(bool gather, const void* src, const int* idx, void* dst, int B, int N, int n_sel, int D,
                      int dtype, cudaStream_t s) {
   const long long row_bytes = (long long)D * dtype_size(dtype);

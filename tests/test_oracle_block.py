@@ -187,6 +187,65 @@ def test_refresh_touches_only_selected_rows_and_reads_the_full_kv_cache():
     assert np.array_equal(orc2.blocks[0].k_cache, st.k_cache)
 
 
+def _one_cached_refresh(cfg, w, poke=None):
+    """One full refresh, an optional change of cached K/V rows, then one cached refresh: (oracle, rows, x_out)."""
+    rng = np.random.default_rng(12)
+    x0, temb0 = rng.standard_normal((2, cfg.n_rows, 32)), rng.standard_normal((2, 12))
+    x1, temb1 = rng.standard_normal((2, cfg.n_rows, 32)), rng.standard_normal((2, 12))
+    orc = O.HeroOracle(cfg, w)
+    orc.block_refresh(0, x0, temb0, None)
+    rows = orc.select(0)
+    if poke is not None:
+        for r in poke(rows):
+            orc.blocks[0].k_cache[:, r] += 0.7
+            orc.blocks[0].v_cache[:, r] -= 0.4
+    return orc, rows, orc.block_refresh(0, x1, temb1, rows)
+
+
+def test_literal_eq3_attention_sees_only_refreshed_and_text_rows():
+    """attend_mode 1: the branch outputs of a cached step do not depend on the cached K/V of video rows that are
+    not refreshed, do depend on the text rows' K/V, and with every video row refreshed equal the default mode
+    (softmax attention does not depend on the order of the keys)."""
+    w = rand_weights(small_cfg(n_blocks=1, n_shallow=1), seed=10)
+    lit = small_cfg(n_blocks=1, n_shallow=1, attend_mode=1)
+    dflt = small_cfg(n_blocks=1, n_shallow=1)
+    stale = lambda rows: np.setdiff1d(np.arange(lit.n_text, lit.n_rows), rows)[:5]
+    text = lambda rows: [1]
+    base = _one_cached_refresh(lit, w)
+    rows = base[1]
+    assert 0 < len(rows) < lit.n_video
+    got = _one_cached_refresh(lit, w, stale)
+    assert np.array_equal(got[2][:, rows], base[2][:, rows])                  # stale video rows are never read
+    got = _one_cached_refresh(lit, w, text)
+    assert np.abs(got[2][:, rows] - base[2][:, rows]).max() > 1e-3            # the text rows are
+    d0, d1 = _one_cached_refresh(dflt, w), _one_cached_refresh(dflt, w, stale)
+    assert np.abs(d1[2][:, rows] - d0[2][:, rows]).max() > 1e-3               # the default mode reads them
+    assert np.abs(d0[2][:, rows] - base[2][:, rows]).max() > 1e-3             # so the two modes differ ...
+    # ... except when nothing is left out
+    w1 = rand_weights(small_cfg(n_blocks=1, n_shallow=1), seed=3)
+    a = _one_cached_refresh(small_cfg(n_blocks=1, n_shallow=1, ratio_den=1, attend_mode=1), w1)
+    b = _one_cached_refresh(small_cfg(n_blocks=1, n_shallow=1, ratio_den=1), w1)
+    assert len(a[1]) == lit.n_video
+    np.testing.assert_allclose(a[2], b[2], rtol=1e-11, atol=1e-12)
+    # one refreshed row by hand: softmax over [text rows, refreshed rows] of the merged cache only
+    orc, rows, _ = base
+    st = orc.blocks[0]
+    rng = np.random.default_rng(12)
+    rng.standard_normal((2, lit.n_rows, 32)); rng.standard_normal((2, 12))
+    x1, temb1 = rng.standard_normal((2, lit.n_rows, 32)), rng.standard_normal((2, 12))
+    bi, r = 0, rows[1]
+    mod = O.modulation(lit, orc.w[0], temb1)
+    q = (O.layernorm_modulate(lit, x1[bi, [r]], mod[0][bi], mod[1][bi]) @ orc.w[0]["w_qkv"].T + orc.w[0]["b_qkv"])[0, :32]
+    seen = list(range(lit.n_text)) + list(rows)
+    out = np.zeros(32)
+    for hd in range(lit.n_heads):
+        sl = slice(hd * lit.head_dim, (hd + 1) * lit.head_dim)
+        sc = np.array([q[sl] @ st.k_cache[bi, j, sl] for j in seen]) / np.sqrt(lit.head_dim)
+        p = np.exp(sc - sc.max()); p /= p.sum()
+        out[sl] = sum(pj * st.v_cache[bi, j, sl] for pj, j in zip(p, seen))
+    np.testing.assert_allclose(st.g[0][bi, r], out @ orc.w[0]["w_o"].T + orc.w[0]["b_o"], rtol=1e-10, atol=1e-12)
+
+
 # ---------------------------------------------------------------- extrapolation (Eq. 5)
 def test_extrapolation_is_exact_on_features_linear_in_step():
     rng = np.random.default_rng(13)
