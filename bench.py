@@ -224,7 +224,10 @@ def build_device_weights(cfg, device):
     for l in range(cfg["n_blocks"]):
         blk = {}
         for name, shape in S.weight_shapes(cfg).items():
-            blk[name] = S.device_normal(cfg["seed"], name, shape, 0.02, l, None, device).to(dt).contiguous()
+            t = S.device_normal(cfg["seed"], name, shape, 0.02, l, None, device)
+            if name in ("qn_w", "kn_w"):
+                t = t + 1.0                       # LayerNorm gains sit around one
+            blk[name] = t.to(dt).contiguous()
         weights.append(blk)
     return weights
 
@@ -347,8 +350,8 @@ def run_hero(args, cfg, rank, world, local_rank):
     hero.close()
 
     # the same cached step under two opt-in variants (reported beside the headline, never as it)
-    def time_variant(extra):
-        hv = H.Hero(dict(run_cfg, **extra), weights)
+    def time_variant(extra, w=None):
+        hv = H.Hero(dict(run_cfg, **extra), w or weights)
         for s_ in range(2):
             hv.hero_step(s_, x, tembs[s_])
         st = 2
@@ -369,7 +372,7 @@ def run_hero(args, cfg, rank, world, local_rank):
         hv.close()
         return out
 
-    collapsed = attend_refreshed = None
+    collapsed = attend_refreshed = base_qk = None
     if not args.no_collapse:
         if cfg["n_shallow"] < cfg["n_blocks"]:
             collapsed = time_variant(dict(deep_collapse=1))
@@ -378,6 +381,13 @@ def run_hero(args, cfg, rank, world, local_rank):
             attend_refreshed = time_variant(dict(attend_mode=1))
             attend_refreshed["note"] = ("attend_mode=1: the refreshed queries of a cached step attend to the refreshed "
                                         "and text rows only (Eq. 3 read literally) instead of the full cached K/V")
+            hd = cfg["head_dim"]
+            w_qk = [dict(blk, qn_w=torch.ones(hd, device=device, dtype=dt), qn_b=torch.zeros(hd, device=device, dtype=dt),
+                         kn_w=torch.ones(hd, device=device, dtype=dt), kn_b=torch.zeros(hd, device=device, dtype=dt))
+                    for blk in weights]
+            base_qk = time_variant(dict(qk_norm=1, rope=1), w_qk)
+            base_qk["note"] = ("qk_norm=1, rope=1: the base model's per-head LayerNorm and 3-D rotary embedding of the "
+                               "fresh q and k rows (one extra HBM-bound pass per refresh block)")
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -409,6 +419,8 @@ def run_hero(args, cfg, rank, world, local_rank):
             line["deep_collapse_variant"] = collapsed
         if attend_refreshed:
             line["attend_refreshed_variant"] = attend_refreshed
+        if base_qk:
+            line["qk_norm_rope_variant"] = base_qk
         if roofline:
             line["roofline"] = roofline
         if cpu_baseline:

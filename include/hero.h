@@ -70,14 +70,25 @@ typedef struct hero_config {
   int attend_mode;         /* which keys the refreshed queries of a cached step attend to: 0 = the full cached
                               K/V of all rows (default); 1 = only the rows refreshed in this step plus the
                               text rows (Eq. 3 read literally, F(S(z), S(tau)) with the text kept) */
+  int qk_norm;             /* 1: LayerNorm (eps 1e-6) of every head's q and k features with the learned gain and
+                              bias qn_w/qn_b, kn_w/kn_b of hero_block_weights, before attention (base-model
+                              detail; the paper's Sec. 3 leaves the block's internals to the base model) */
+  int rope;                /* 1: 3-D rotary embedding of the video rows' q and k (after qk_norm): head feature
+                              pairs (2i, 2i+1); with P = head_dim/2 pairs, the first P/4 turn with the frame
+                              index, the next (P - P/4)/2 with the grid row, the rest with the grid column,
+                              pair i of an axis with n pairs by pos * 10000^(-i/n) radians; text rows are
+                              not turned.  The K cache holds keys in this final form. */
 } hero_config;
 
 /* Device pointers to one block's parameters (borrowed for the context's lifetime).
  * w_mod [n_mod*hidden, temb_dim] with chunks (shift1, scale1, shift2, scale2[, gate1, gate2]);
  * w_qkv [3*hidden, hidden] with output chunks (q, k, v); w_o [hidden, hidden];
- * w_1 [ffn_dim, hidden]; w_2 [hidden, ffn_dim]; biases match the output size. */
+ * w_1 [ffn_dim, hidden]; w_2 [hidden, ffn_dim]; biases match the output size.
+ * qn_w, qn_b, kn_w, kn_b [head_dim] (run dtype): gains and biases of the q/k LayerNorm, shared by the
+ * heads; read only when hero_config.qk_norm is 1, NULL otherwise. */
 typedef struct hero_block_weights {
   const void *w_mod, *b_mod, *w_qkv, *b_qkv, *w_o, *b_o, *w_1, *b_1, *w_2, *b_2;
+  const void *qn_w, *qn_b, *kn_w, *kn_b;
 } hero_block_weights;
 
 /* ---- context ------------------------------------------------------------- */

@@ -64,8 +64,12 @@ class Config:
     track_mode: int = 0       # 0: weighted draw (age+1)*(hash+1); 1: strict oldest-first (age, hash)
     share_selection: int = 0  # 1: one list per cached step (block 0's sampler) for every shallow block
     attend_mode: int = 0      # 0: refreshed queries see the full cached K/V; 1: refreshed + text rows only
+    qk_norm: int = 0          # 1: per-head LayerNorm (learned affine) of q and k before attention
+    rope: int = 0             # 1: 3-D rotary position embedding of the video rows' q and k
     seed: int = 0
     eps: float = 1e-5
+    qk_eps: float = 1e-6
+    rope_theta: float = 10000.0
 
     @classmethod
     def from_dict(cls, d):
@@ -215,6 +219,68 @@ def layernorm_modulate(cfg: Config, x, shift, scale):
     return (x - mu) / np.sqrt(var + cfg.eps) * (1.0 + scale) + shift
 
 
+def qk_layernorm(cfg: Config, t, gamma, beta):
+    """LayerNorm of every head's slice of t [n, D] over its head_dim features (biased
+    variance, eps = qk_eps), times gamma plus beta (both [head_dim], shared by the heads).
+    The base model normalises q and k this way before attention; the paper leaves the
+    block's internals to the base model (Sec. 3)."""
+    n = t.shape[0]
+    th = t.reshape(n, cfg.n_heads, cfg.head_dim)
+    mu = th.mean(axis=-1, keepdims=True)
+    var = ((th - mu) ** 2).mean(axis=-1, keepdims=True)
+    return ((th - mu) / np.sqrt(var + cfg.qk_eps) * gamma + beta).reshape(n, cfg.hidden)
+
+
+def rope_sections(cfg: Config):
+    """Number of rotary pairs given to the (frame, height, width) axes: a quarter of the
+    head's pairs to time, the rest split evenly over the two spatial axes (8, 12, 12 pairs
+    = 16, 24, 24 features at head_dim 64)."""
+    pairs = cfg.head_dim // 2
+    p_t = pairs // 4
+    p_h = (pairs - p_t) // 2
+    return p_t, p_h, pairs - p_t - p_h
+
+
+def rope_angles(cfg: Config, rows):
+    """Rotation angle of every rotary pair for sequence rows `rows`: [len(rows), head_dim/2].
+    A video token at grid position (f, y, x) turns pair i of an axis' section by
+    pos * theta^(-i / pairs_of_that_axis); text rows (the first n_text) are not turned."""
+    rows = np.asarray(rows)
+    ang = np.zeros((len(rows), cfg.head_dim // 2), F64)
+    v = rows - cfg.n_text
+    is_video = v >= 0
+    v = np.where(is_video, v, 0)
+    pos = (v // (cfg.grid_h * cfg.grid_w), (v // cfg.grid_w) % cfg.grid_h, v % cfg.grid_w)
+    at = 0
+    for axis, n_pairs in enumerate(rope_sections(cfg)):
+        for i in range(n_pairs):
+            ang[:, at + i] = pos[axis] * cfg.rope_theta ** (-i / n_pairs)
+        at += n_pairs
+    return ang * is_video[:, None]
+
+
+def apply_rope(cfg: Config, t, rows):
+    """Rotate the feature pairs (2i, 2i+1) of every head of t [len(rows), D] by rope_angles."""
+    n = t.shape[0]
+    ang = rope_angles(cfg, rows)[:, None, :]                      # the same for every head
+    th = t.reshape(n, cfg.n_heads, cfg.head_dim // 2, 2)
+    even, odd = th[..., 0], th[..., 1]
+    out = np.stack([even * np.cos(ang) - odd * np.sin(ang), even * np.sin(ang) + odd * np.cos(ang)], axis=-1)
+    return out.reshape(n, cfg.hidden)
+
+
+def prepare_qk(cfg: Config, w, q, k, rows):
+    """The base model's treatment of q and k between the QKV projection and attention:
+    optional per-head LayerNorm, then optional rotary embedding by the rows' positions.
+    K is cached in this final form, which stays valid because a row never moves."""
+    if cfg.qk_norm:
+        q = qk_layernorm(cfg, q, w["qn_w"], w["qn_b"])
+        k = qk_layernorm(cfg, k, w["kn_w"], w["kn_b"])
+    if cfg.rope:
+        q, k = apply_rope(cfg, q, rows), apply_rope(cfg, k, rows)
+    return q, k
+
+
 def attention(cfg: Config, q, k_all, v_all):
     """softmax(q K^T / sqrt(head_dim)) V per head, queries [n, D] against all rows
     of K, V [N, D]; no mask.  The score matrix of one head is formed here only
@@ -323,6 +389,7 @@ class HeroOracle:
             a = layernorm_modulate(c, x[b, rows], shift1[b], scale1[b])
             qkv = a @ w["w_qkv"].T + w["b_qkv"]
             q, k, v = qkv[:, :D], qkv[:, D:2 * D], qkv[:, 2 * D:]
+            q, k = prepare_qk(c, w, q, k, rows)
             st.k_cache[b, rows] = k
             st.v_cache[b, rows] = v
             sel = np.searchsorted(rows, rows_out)
@@ -423,6 +490,16 @@ def uncached_forward(cfg: Config, weights, x, temb):
                 qh = qkv[:, h * hd:(h + 1) * hd]
                 kh = qkv[:, D + h * hd:D + (h + 1) * hd]
                 vh = qkv[:, 2 * D + h * hd:2 * D + (h + 1) * hd]
+                if cfg.qk_norm:
+                    qh = (qh - qh.mean(-1, keepdims=True)) / np.sqrt(qh.var(-1, keepdims=True) + cfg.qk_eps) * w["qn_w"] + w["qn_b"]
+                    kh = (kh - kh.mean(-1, keepdims=True)) / np.sqrt(kh.var(-1, keepdims=True) + cfg.qk_eps) * w["kn_w"] + w["kn_b"]
+                if cfg.rope:
+                    # pairs as complex numbers times e^{i angle}
+                    turn = np.exp(1j * rope_angles(cfg, np.arange(N)))
+                    qh = np.stack([((qh[:, 0::2] + 1j * qh[:, 1::2]) * turn).real,
+                                   ((qh[:, 0::2] + 1j * qh[:, 1::2]) * turn).imag], -1).reshape(N, hd)
+                    kh = np.stack([((kh[:, 0::2] + 1j * kh[:, 1::2]) * turn).real,
+                                   ((kh[:, 0::2] + 1j * kh[:, 1::2]) * turn).imag], -1).reshape(N, hd)
                 s = np.exp(qh @ kh.T / np.sqrt(hd) - (qh @ kh.T / np.sqrt(hd)).max(-1, keepdims=True))
                 heads.append((s / s.sum(-1, keepdims=True)) @ vh)
             ga = np.concatenate(heads, -1) @ w["w_o"].T + w["b_o"]

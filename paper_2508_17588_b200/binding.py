@@ -35,12 +35,14 @@ class HeroConfig(C.Structure):
         "n_blocks", "n_shallow", "hidden", "n_heads", "head_dim", "ffn_dim", "temb_dim",
         "batch", "frames", "grid_h", "grid_w", "n_text", "patch_h", "patch_w",
         "ratio_num", "ratio_den", "quota_mode", "warmup_full_steps", "full_interval", "dtype", "has_gate")
-    ] + [("seed", C.c_ulonglong), ("deep_collapse", C.c_int), ("track_mode", C.c_int), ("share_selection", C.c_int), ("attend_mode", C.c_int)]
+    ] + [("seed", C.c_ulonglong), ("deep_collapse", C.c_int), ("track_mode", C.c_int), ("share_selection", C.c_int), ("attend_mode", C.c_int), ("qk_norm", C.c_int), ("rope", C.c_int)]
 
 
 class HeroBlockWeights(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in
-                ("w_mod", "b_mod", "w_qkv", "b_qkv", "w_o", "b_o", "w_1", "b_1", "w_2", "b_2")]
+                ("w_mod", "b_mod", "w_qkv", "b_qkv", "w_o", "b_o", "w_1", "b_1", "w_2", "b_2",
+                 "qn_w", "qn_b", "kn_w", "kn_b")]
+    OPTIONAL = ("qn_w", "qn_b", "kn_w", "kn_b")      # read only with hero_config.qk_norm
 
 
 class HeroError(RuntimeError):
@@ -159,6 +161,8 @@ class Hero:
         arr = (HeroBlockWeights * cfg["n_blocks"])()
         for l, w in enumerate(weights):
             for name, _ in HeroBlockWeights._fields_:
+                if name in HeroBlockWeights.OPTIONAL and not cfg.get("qk_norm", 0):
+                    continue
                 t = w[name]
                 assert t.is_cuda and t.is_contiguous() and t.dtype == self.dt, name
                 setattr(arr[l], name, t.data_ptr())

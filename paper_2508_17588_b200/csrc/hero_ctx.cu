@@ -1,6 +1,7 @@
 // Context, bookkeeping and the C ABI of the HERO cached step (Algorithm 1).
 // All device work is enqueued on the context's stream; the host only does schedule
 // arithmetic (which step is full, the selection list length, k and d of Eq. 5).
+#include <math.h>
 #include <stdio.h>
 #include <string.h>
 
@@ -49,6 +50,9 @@ struct hero_ctx {
   // attend_mode 1: compact K/V of the rows a cached step attends to (text + refreshed) and their list
   void* kv_cmp[2] = {nullptr, nullptr};
   int* att_list = nullptr;
+  // rope 1: (cos, sin) of every (axis position, rotary pair), computed on the host in double precision
+  float2* rope_tab = nullptr;
+  int rope_pairs[3] = {0, 0, 0};
   void *ws_a = nullptr, *ws_q = nullptr, *ws_o = nullptr, *ws_u = nullptr;
   float* mod = nullptr;                  // [B, n_mod*D] adaLN vectors of the current block
   int* idx_ws = nullptr;                 // [n_shallow, idx_cap] selection lists of the current step
@@ -200,6 +204,17 @@ int refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, const i
   o_qkv.ptr[2] = vdst;    o_qkv.ld[2] = D; o_qkv.scatter[2] = 1;
   o_qkv.seg_cols = D; o_qkv.idx = d_idx; o_qkv.n_sel = n_sel; o_qkv.n_rows = N;
   HERO_TRY(run_gemm(c, c->ws_a, w.w_qkv, w.b_qkv, M, 3 * D, D, o_qkv));
+  if (g.qk_norm || g.rope) {
+    QkPrepArgs qa = {};
+    qa.q = c->ws_q; qa.k = kdst; qa.idx = d_idx;
+    if (g.qk_norm) { qa.qn_w = w.qn_w; qa.qn_b = w.qn_b; qa.kn_w = w.kn_w; qa.kn_b = w.kn_b; }
+    qa.rope = g.rope ? c->rope_tab : nullptr;
+    qa.B = B; qa.N = N; qa.n_sel = n_sel; qa.D = D; qa.n_heads = g.n_heads; qa.head_dim = g.head_dim;
+    qa.n_text = g.n_text; qa.frames = g.frames; qa.grid_h = g.grid_h; qa.grid_w = g.grid_w;
+    qa.p_t = c->rope_pairs[0]; qa.p_h = c->rope_pairs[1]; qa.p_w = c->rope_pairs[2];
+    qa.eps = 1e-6f;
+    HERO_LAUNCH(c, HERO_PROF_GATHER_LN, launch_qk_prep(qa, g.dtype, c->stream));
+  }
   if (g.attend_mode == 1 && !full) {
     // Eq. 3 read literally: the refreshed queries see the refreshed rows (just written) and the text rows
     const int n_att = g.n_text + n_sel;
@@ -291,6 +306,8 @@ int validate(const hero_config* g) {
   if (g->track_mode != 0 && g->track_mode != 1) return HERO_ERR_ARG;
   if (g->share_selection != 0 && g->share_selection != 1) return HERO_ERR_ARG;
   if (g->attend_mode != 0 && g->attend_mode != 1) return HERO_ERR_ARG;
+  if ((g->qk_norm != 0 && g->qk_norm != 1) || (g->rope != 0 && g->rope != 1)) return HERO_ERR_ARG;
+  if ((g->qk_norm || g->rope) && (g->head_dim % 2 != 0 || g->head_dim > 256)) return HERO_ERR_ARG;
   if (g->dtype == HERO_DTYPE_BF16) {
     if (g->head_dim != 64 || g->hidden % 8 || g->ffn_dim % 8 || g->temb_dim % 8) return HERO_ERR_ALIGN;
   } else {
@@ -342,6 +359,12 @@ int hero_init(hero_ctx** out, const hero_config* cfg, const hero_block_weights* 
       if (!p) return HERO_ERR_ARG;
       if (!aligned16(p)) return HERO_ERR_ALIGN;
     }
+    if (cfg->qk_norm) {
+      for (const void* p : {blocks[l].qn_w, blocks[l].qn_b, blocks[l].kn_w, blocks[l].kn_b}) {
+        if (!p) return HERO_ERR_ARG;
+        if (!aligned16(p)) return HERO_ERR_ALIGN;
+      }
+    }
   }
   if (cfg->dtype == HERO_DTYPE_BF16) HERO_TRY(tc_init_driver_api());
   hero_ctx* c = new (std::nothrow) hero_ctx();
@@ -379,6 +402,21 @@ int hero_init(hero_ctx** out, const hero_config* cfg, const hero_block_weights* 
     A(&c->kv_cmp[0], tensor); A(&c->kv_cmp[1], tensor);
     A((void**)&c->att_list, (size_t)c->N * sizeof(int));
   }
+  std::vector<float2> rope_host;
+  if (cfg->rope) {
+    const int pairs = cfg->head_dim / 2;
+    c->rope_pairs[0] = pairs / 4;
+    c->rope_pairs[1] = (pairs - c->rope_pairs[0]) / 2;
+    c->rope_pairs[2] = pairs - c->rope_pairs[0] - c->rope_pairs[1];
+    const int extent[3] = {cfg->frames, cfg->grid_h, cfg->grid_w};
+    for (int ax = 0; ax < 3; ++ax)
+      for (int pos = 0; pos < extent[ax]; ++pos)
+        for (int i = 0; i < c->rope_pairs[ax]; ++i) {
+          const double ang = (double)pos * std::pow(10000.0, -(double)i / (double)c->rope_pairs[ax]);
+          rope_host.push_back(make_float2((float)std::cos(ang), (float)std::sin(ang)));
+        }
+    A((void**)&c->rope_tab, (rope_host.size() + 1) * sizeof(float2));
+  }
   A(&c->ws_a, tensor); A(&c->ws_q, tensor); A(&c->ws_o, tensor);
   A(&c->ws_u, (size_t)cfg->batch * c->N * cfg->ffn_dim * c->esz);
   A((void**)&c->mod, (size_t)cfg->batch * c->n_mod * cfg->hidden * sizeof(float));
@@ -387,6 +425,10 @@ int hero_init(hero_ctx** out, const hero_config* cfg, const hero_block_weights* 
   A(&c->x_stage, tensor);
   A(&c->temb_stage, (size_t)cfg->batch * cfg->temb_dim * c->esz);
   if (rc != HERO_OK) { hero_destroy(c); return rc; }
+  if (!rope_host.empty()) {
+    cudaError_t er = cudaMemcpy(c->rope_tab, rope_host.data(), rope_host.size() * sizeof(float2), cudaMemcpyHostToDevice);
+    if (er != cudaSuccess) { set_cuda_error(er, "cudaMemcpy(rope table)"); hero_destroy(c); return HERO_ERR_CUDA; }
+  }
   cudaError_t e = cudaMemsetAsync(c->d_status, 0, 16, c->stream);
   if (e != cudaSuccess) { set_cuda_error(e, "cudaMemsetAsync"); hero_destroy(c); return HERO_ERR_CUDA; }
   rc = hero_reset(c);

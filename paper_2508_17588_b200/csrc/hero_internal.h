@@ -84,6 +84,19 @@ int launch_residual2(void* x, const void* ga, const void* gf, long long n, int d
 int launch_residual2_acc(void* x, const void* ga, const void* gf, float* acc, long long n, int dtype, cudaStream_t s);
 int launch_extrapolate_stack(void* x, const float* s_prev, const float* s_last, long long n, int k, int d, int dtype,
                              cudaStream_t s);
+// Per-head LayerNorm and rotary embedding of fresh q (compact) and k (in the cache) rows.
+struct QkPrepArgs {
+  void* q;                 // [B, n_sel, D]
+  void* k;                 // [B, N, D], rows idx[i] (or i when idx is null)
+  const int* idx;
+  const void *qn_w, *qn_b, *kn_w, *kn_b;   // [head_dim] in the run dtype, or all null
+  const float2* rope;      // (cos, sin) per (axis position, pair) or null
+  int B, N, n_sel, D, n_heads, head_dim;
+  int n_text, frames, grid_h, grid_w;
+  int p_t, p_h, p_w;       // rotary pairs per axis
+  float eps;
+};
+int launch_qk_prep(const QkPrepArgs& a, int dtype, cudaStream_t s);
 // list[i] = i for i < n_text, list[n_text + i] = idx[i] for i < n_sel (rows a literal Eq. 3 attends to)
 int launch_attend_list(const int* idx, int n_sel, int n_text, int* list, cudaStream_t s);
 int launch_gather_rows(const void* src, const int* idx, void* dst, int B, int N, int n_sel, int D,

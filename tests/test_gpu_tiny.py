@@ -176,11 +176,12 @@ def test_paper_hyperparameters_small_model():
 
 
 @pytest.mark.parametrize("variant", [dict(track_mode=1), dict(share_selection=1), dict(track_mode=1, share_selection=1, deep_collapse=1),
-                                     dict(attend_mode=1), dict(attend_mode=1, share_selection=1, quota_mode=1)])
+                                     dict(attend_mode=1), dict(attend_mode=1, share_selection=1, quota_mode=1),
+                                     dict(qk_norm=1), dict(rope=1), dict(qk_norm=1, rope=1, attend_mode=1, has_gate=1)])
 def test_tracking_and_selection_variants(variant):
     """Strict oldest-first tracking, one selection list shared by all refresh blocks of a step, both together
-    with the collapsed deep stack, and attention restricted to the refreshed and text rows: 8 steps through
-    hero_step against the oracle."""
+    with the collapsed deep stack, attention restricted to the refreshed and text rows, and the base model's
+    q/k LayerNorm and rotary embedding: 8 steps through hero_step against the oracle."""
     cfgd = dict(S.CONFIGS["tiny"], n_blocks=5, n_shallow=3, full_interval=3, steps=8, seed=21, **variant)
     orc, hero, _ = make_pair(cfgd)
     x_host = S.tokens(cfgd)

@@ -25,8 +25,8 @@ def small_cfg(**kw):
 def rand_weights(cfg, scale=0.2, seed=0):
     rng = np.random.default_rng(seed)
     d = dict(cfg.__dict__, dtype="fp32")
-    return [{k: rng.standard_normal(shp) * scale for k, shp in S.weight_shapes(d).items()}
-            for _ in range(cfg.n_blocks)]
+    return [{k: rng.standard_normal(shp) * scale + (1.0 if k in ("qn_w", "kn_w") else 0.0)
+             for k, shp in S.weight_shapes(d).items()} for _ in range(cfg.n_blocks)]
 
 
 def t64(a):
@@ -115,11 +115,55 @@ def test_full_block_vs_torch_library_block(gate):
     np.testing.assert_allclose(st.v_cache, v, rtol=1e-10, atol=1e-11)
 
 
-# ---------------------------------------------------------------- cached == uncached where the paper says so
-def test_ratio_one_without_extrapolation_equals_uncached_step():
+# ---------------------------------------------------------------- q/k LayerNorm and rotary embedding
+def test_qk_layernorm_vs_torch_layer_norm_per_head():
+    cfg = small_cfg(qk_norm=1)
+    rng = np.random.default_rng(30)
+    t = rng.standard_normal((7, cfg.hidden)) * 3 + 1
+    gamma, beta = rng.standard_normal(cfg.head_dim), rng.standard_normal(cfg.head_dim)
+    got = O.qk_layernorm(cfg, t, gamma, beta)
+    want = TF.layer_norm(t64(t).reshape(7, cfg.n_heads, cfg.head_dim), (cfg.head_dim,), t64(gamma), t64(beta),
+                         eps=1e-6).reshape(7, cfg.hidden).numpy()
+    np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-12)
+
+
+def test_rope_fixed_points_known_angles_and_shift_invariance():
+    cfg = small_cfg(rope=1, head_dim=16, n_heads=2, frames=4, grid_h=6, grid_w=8)     # 8 pairs: 2 + 3 + 3
+    assert O.rope_sections(cfg) == (2, 3, 3)
+    assert O.rope_sections(small_cfg(head_dim=64, hidden=128)) == (8, 12, 12)          # 16 + 24 + 24 features
+    row = lambda f, y, x: cfg.n_text + (f * cfg.grid_h + y) * cfg.grid_w + x
+    rng = np.random.default_rng(31)
+    t = rng.standard_normal((4, cfg.hidden))
+    rows = np.array([1, row(0, 0, 0), row(2, 3, 4), row(3, 5, 7)])
+    got = O.apply_rope(cfg, t, rows)
+    assert np.array_equal(got[0], t[0])                         # a text row is not turned
+    np.testing.assert_allclose(got[1], t[1], atol=1e-15)        # nor is the video token at the origin
+    pairs = lambda a: a.reshape(-1, cfg.n_heads, 8, 2)
+    np.testing.assert_allclose(np.linalg.norm(pairs(got), axis=-1), np.linalg.norm(pairs(t), axis=-1), rtol=1e-12)
+    # unit vectors along the even feature of a pair come out as (cos, sin) of that pair's angle
+    e = np.zeros((1, cfg.hidden)); e[0, 0::2] = 1.0
+    turned = pairs(O.apply_rope(cfg, e, np.array([row(2, 3, 4)])))[0]
+    want_angle = np.array([2.0, 2.0 * 10000 ** (-1 / 2),                          # frame axis, 2 pairs
+                           3.0, 3.0 * 10000 ** (-1 / 3), 3.0 * 10000 ** (-2 / 3),  # grid row, 3 pairs
+                           4.0, 4.0 * 10000 ** (-1 / 3), 4.0 * 10000 ** (-2 / 3)])
+    for h in range(cfg.n_heads):
+        np.testing.assert_allclose(turned[h, :, 0], np.cos(want_angle), rtol=1e-12, atol=1e-15)
+        np.testing.assert_allclose(turned[h, :, 1], np.sin(want_angle), rtol=1e-12, atol=1e-15)
+    # scores depend on the displacement between query and key, not on where the pair sits
+    q, k = rng.standard_normal((1, cfg.hidden)), rng.standard_normal((1, cfg.hidden))
+    dot = lambda a, b: (O.apply_rope(cfg, q, np.array([a])) @ O.apply_rope(cfg, k, np.array([b])).T).item()
+    base = dot(row(1, 2, 3), row(0, 1, 5))
+    assert abs(dot(row(3, 4, 4), row(2, 3, 6)) - base) < 1e-12
+    assert abs(dot(row(1, 2, 3), row(0, 1, 6)) - base) > 1e-3
+
+
+@pytest.mark.parametrize("extras", [dict(), dict(qk_norm=1, rope=1)])
+def test_ratio_one_without_extrapolation_equals_uncached_step(extras):
     """R = 1 makes S(z) = z; with text rows included and every block shallow, a cached
-    step is Eq. 2 on all rows, i.e. the uncached forward, on every step."""
-    cfg = small_cfg(n_blocks=3, n_shallow=3, ratio_num=1, ratio_den=1)
+    step is Eq. 2 on all rows, i.e. the uncached forward, on every step.  With q/k LayerNorm and
+    rotary embedding on, the uncached forward normalises with numpy's var and turns the pairs as
+    complex numbers, the block path by the plain real formulas."""
+    cfg = small_cfg(n_blocks=3, n_shallow=3, ratio_num=1, ratio_den=1, **extras)
     w = rand_weights(cfg, seed=5)
     rng = np.random.default_rng(6)
     orc = O.HeroOracle(cfg, w)

@@ -109,18 +109,29 @@ def weight_shapes(cfg) -> dict:
     """All weight matrices are row-major [out_features, in_features]."""
     D, F, E = cfg["hidden"], cfg["ffn_dim"], cfg["temb_dim"]
     n_mod = 6 if cfg.get("has_gate", 0) else 4
-    return {"w_mod": (n_mod * D, E), "b_mod": (n_mod * D,),
-            "w_qkv": (3 * D, D), "b_qkv": (3 * D,),
-            "w_o": (D, D), "b_o": (D,),
-            "w_1": (F, D), "b_1": (F,),
-            "w_2": (D, F), "b_2": (D,)}
+    shapes = {"w_mod": (n_mod * D, E), "b_mod": (n_mod * D,),
+              "w_qkv": (3 * D, D), "b_qkv": (3 * D,),
+              "w_o": (D, D), "b_o": (D,),
+              "w_1": (F, D), "b_1": (F,),
+              "w_2": (D, F), "b_2": (D,)}
+    if cfg.get("qk_norm", 0):
+        hd = cfg["head_dim"]
+        shapes.update({"qn_w": (hd,), "qn_b": (hd,), "kn_w": (hd,), "kn_b": (hd,)})
+    return shapes
 
 
 def block_weights(cfg, block: int) -> dict:
     """Weights of one block, N(0, 0.02), as fp32 arrays (bf16-exact if cfg is bf16)."""
     out = {}
     for name, shape in weight_shapes(cfg).items():
-        out[name] = normal(cfg["seed"], name, shape, std=0.02, index=block, dtype=cfg["dtype"])
+        if name in ("qn_w", "kn_w"):       # LayerNorm gains: around one
+            out[name] = 1.0 + normal(cfg["seed"], name, shape, std=0.1, index=block)
+        elif name in ("qn_b", "kn_b"):
+            out[name] = normal(cfg["seed"], name, shape, std=0.1, index=block)
+        else:
+            out[name] = normal(cfg["seed"], name, shape, std=0.02, index=block, dtype=cfg["dtype"])
+        if cfg["dtype"] == "bf16":
+            out[name] = round_bf16(out[name])
     return out
 
 
