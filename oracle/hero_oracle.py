@@ -470,6 +470,37 @@ class HeroOracle:
 # =============================================================================
 # The uncached step (Eq. 2 applied to every row, nothing stored)
 # =============================================================================
+# =============================================================================
+# Diagnostics (Sec. 4.1, hierarchical feature analysis; Fig. 4)
+# =============================================================================
+def second_difference_variance(features):
+    """Variance, over all steps and elements, of the second-order temporal differences
+    F_{t+1} - 2 F_t + F_{t-1} of one layer's features.  features: [T, ...] with T >= 3."""
+    f = np.asarray(features, F64)
+    d2 = f[2:] - 2.0 * f[1:-1] + f[:-2]
+    return float(np.mean((d2 - d2.mean()) ** 2))
+
+
+def stability_scores(per_layer_features):
+    """Stability score of every layer in [0, 1], higher = more stable (Sec. 4.1): the
+    variances of the second-order differences are min-max normalised over the layers and
+    inverted, so the layer whose features fluctuate most gets 0 and the steadiest gets 1.
+    The paper states the range and the direction only; min-max over the layers is this
+    reading.  All-equal variances give 1 everywhere."""
+    v = np.array([second_difference_variance(f) for f in per_layer_features], F64)
+    span = v.max() - v.min()
+    if span == 0.0:
+        return np.ones_like(v)
+    return 1.0 - (v - v.min()) / span
+
+
+def extrapolation_error(g_prev, g_last, g_true, k: int, d: int):
+    """Relative L2 error of Eq. 5's prediction against the features actually computed k
+    steps after g_last: ||extrap - g_true|| / ||g_true||."""
+    e = extrapolate(np.asarray(g_prev, F64), np.asarray(g_last, F64), k, d) - np.asarray(g_true, F64)
+    return float(np.sqrt((e ** 2).sum() / (np.asarray(g_true, F64) ** 2).sum()))
+
+
 def uncached_forward(cfg: Config, weights, x, temb):
     """Plain DiT block stack with no cache at all; written separately from
     HeroOracle so that "refresh ratio 1 with extrapolation off" can be checked

@@ -428,3 +428,48 @@ def test_deep_stack_extrapolate_matches_block_by_block_step():
     b.block_refresh(0, xb, S.temb(cfgd, 2), rows)
     b.deep_stack_extrapolate(xb, 1, 1)
     assert np.allclose(xa, xb, rtol=0, atol=1e-11)
+
+
+# ---------------------------------------------------------------- diagnostics (Sec. 4.1)
+def test_second_difference_variance_closed_forms():
+    rng = np.random.default_rng(40)
+    a, b, c = rng.standard_normal((3, 5, 7))
+    t = np.arange(6.0)[:, None, None]
+    assert O.second_difference_variance(a + b * t) < 1e-24                      # linear in the step: no curvature
+    # quadratic in the step: the second difference is 2c at every step, so its variance is that of 2c over elements
+    np.testing.assert_allclose(O.second_difference_variance(a + b * t + c * t * t), np.var(2 * c), rtol=1e-10)
+    # white noise of variance s^2 per step: coefficients (1, -2, 1) give 6 s^2
+    f = rng.standard_normal((400, 2000)) * 0.5
+    np.testing.assert_allclose(O.second_difference_variance(f), 6 * 0.25, rtol=2e-2)
+    # brute force on a tiny input
+    g = rng.standard_normal((4, 3))
+    d2 = [g[t + 1][j] - 2 * g[t][j] + g[t - 1][j] for t in (1, 2) for j in range(3)]
+    np.testing.assert_allclose(O.second_difference_variance(g), np.var(d2), rtol=1e-12)
+
+
+def test_stability_scores_order_range_and_invariances():
+    rng = np.random.default_rng(41)
+    noise = rng.standard_normal((3, 8, 50))
+    layers = [noise[0] * 2.0, noise[1] * 0.5, noise[2] * 1.0]                   # most, least, middling fluctuation
+    sc = O.stability_scores(layers)
+    assert sc[0] == 0.0 and sc[1] == 1.0 and 0.0 < sc[2] < 1.0
+    v = [O.second_difference_variance(f) for f in layers]
+    np.testing.assert_allclose(sc[2], 1.0 - (v[2] - v[1]) / (v[0] - v[1]), rtol=1e-12)
+    # a drift that is linear in the step changes nothing; a common rescaling of all layers neither
+    t = np.arange(8.0)[:, None]
+    np.testing.assert_allclose(O.stability_scores([f + 3.0 * t + 1.0 for f in layers]), sc, atol=1e-12)
+    np.testing.assert_allclose(O.stability_scores([7.0 * f for f in layers]), sc, atol=1e-12)
+    assert np.array_equal(O.stability_scores([layers[0], layers[0]]), np.ones(2))
+
+
+def test_extrapolation_error_is_zero_on_linear_features_and_known_on_a_quadratic():
+    rng = np.random.default_rng(42)
+    a, b, c = rng.standard_normal((3, 4, 6))
+    f = lambda t: a + b * t + c * t * t
+    lin = lambda t: a + b * t
+    assert O.extrapolation_error(lin(0.0), lin(5.0), lin(7.0), 2, 5) < 1e-14
+    # features quadratic in the step, sampled at 0 and d, predicted at d + k: the line through the two samples
+    # misses by c k (d + k), whatever a and b are
+    d, k = 5, 2
+    want = np.linalg.norm(c * k * (d + k)) / np.linalg.norm(f(d + k))
+    np.testing.assert_allclose(O.extrapolation_error(f(0.0), f(float(d)), f(float(d + k)), k, d), want, rtol=1e-12)
