@@ -504,6 +504,14 @@ def run_kernels(args):
         ms = _time_flushed(lambda: H.hero_extrapolate(a, b_, o, 4, 5), iters, warm, flush)
         hbm("extrapolate", ms, 3 * a.numel() * 2)
         del a, b_, o
+    if want("diagnostics"):
+        a, b_, c_ = rnd(B, N, D), rnd(B, N, D), rnd(B, N, D)
+        mom = torch.zeros(2, dtype=torch.float64, device=dev)
+        ms = _time_flushed(lambda: H.hero_second_difference_moments(a, b_, c_, mom), iters, warm, flush)
+        hbm("second_difference_moments", ms, 3 * a.numel() * 2)
+        ms = _time_flushed(lambda: H.hero_extrapolation_error(a, b_, c_, 2, 5, mom), iters, warm, flush)
+        hbm("extrapolation_error", ms, 3 * a.numel() * 2)
+        del a, b_, c_
     if want("gather") or want("scatter"):
         src = rnd(B, N, D)
         for key, idx in lists.items():
@@ -591,7 +599,7 @@ def main():
     ap.add_argument("--impl", default="hero", choices=["hero", "reference"])
     ap.add_argument("--workload", default="dit42", choices=["dit42", "aether", "paper_hp", "tiny", "kernels"])
     ap.add_argument("--only", default="", help="kernels workload: comma list of select,extrapolate,gather,scatter,"
-                                               "attention,gemm,deep,block")
+                                               "attention,gemm,deep,block,diagnostics")
     ap.add_argument("--small", action="store_true", help="kernels workload: profiler-sized tensor-core cases")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-collapse", action="store_true", help="skip the variant runs (collapsed deep stack, refreshed-rows-only attention)")

@@ -174,6 +174,24 @@ int hero_step_host(hero_ctx *ctx, int step, void *h_x, const void *h_temb);
 /* 1 if hero_step would run `step` as a full step. */
 int hero_is_full_step(const hero_ctx *ctx, int step);
 
+/* ---- diagnostics (Sec. 4.1, hierarchical feature analysis; stateless) ------- */
+
+/* Moments of the second-order temporal difference u = f_a - 2 f_b + f_c of one layer's features at
+ * three consecutive steps: d_moments[0] += sum u, d_moments[1] += sum u^2 (device doubles, 8-byte
+ * aligned, zeroed by the caller; calls accumulate, so a run over T steps adds T-2 calls per layer).
+ * The variance of the paper's analysis is m1/n - (m0/n)^2 over the n elements summed; its [0, 1]
+ * stability score is the min-max normalisation of these variances over the layers, inverted.
+ * Tensors: n_elem elements of the given dtype, 16-byte aligned.  The sums are formed in double
+ * precision from fp32 partial sums of at most 512 elements; the order of the block sums is not
+ * fixed, so results repeat to about 1e-15 relative, not bit for bit. */
+int hero_second_difference_moments(const void *d_f_a, const void *d_f_b, const void *d_f_c, long long n_elem,
+                                   int dtype, double *d_moments, void *stream);
+/* Squared error of Eq. 5 against the truth: with e = g_last + (g_last - g_prev) * k/d,
+ * d_err[0] += sum (e - g_true)^2 and d_err[1] += sum g_true^2; sqrt(d_err[0] / d_err[1]) is the
+ * relative L2 error of extrapolating k steps from two full steps d apart.  Same conventions. */
+int hero_extrapolation_error(const void *d_g_prev, const void *d_g_last, const void *d_g_true, long long n_elem,
+                             int k, int d, int dtype, double *d_err, void *stream);
+
 /* ---- isolated kernels (stateless; stream = cudaStream_t) ------------------- */
 
 /* Eq. 5 alone: out = g_last + (g_last - g_prev) * k/d over n_elem elements. */

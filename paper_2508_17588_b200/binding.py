@@ -26,7 +26,7 @@ EXPORTS = [
     "hero_device_bytes", "hero_launch_count", "hero_profile_begin", "hero_profile_end", "hero_select_tokens", "hero_next_n_sel", "hero_refresh_block",
     "hero_extrapolate_block", "hero_extrapolate_deep_stack", "hero_step", "hero_step_host", "hero_is_full_step", "hero_extrapolate",
     "hero_gather_rows", "hero_scatter_rows", "hero_gemm_bf16", "hero_attention_bf16", "hero_attention_bf16_static", "hero_isolated_status",
-    "hero_state_get", "hero_state_set",
+    "hero_state_get", "hero_state_set", "hero_second_difference_moments", "hero_extrapolation_error",
 ]
 
 
@@ -93,6 +93,8 @@ def load() -> C.CDLL:
         "hero_attention_bf16": (i, [vp, vp, vp, vp, i, i, i, i, vp]),
         "hero_attention_bf16_static": (i, [vp, vp, vp, vp, i, i, i, i, vp, ip]),
         "hero_isolated_status": (i, [vp]),
+        "hero_second_difference_moments": (i, [vp, vp, vp, ll, i, vp, vp]),
+        "hero_extrapolation_error": (i, [vp, vp, vp, ll, i, i, i, vp, vp]),
         "hero_state_get": (i, [vp, i, i, vp, ll]),
         "hero_state_set": (i, [vp, i, i, vp, ll]),
     }
@@ -264,6 +266,25 @@ def hero_extrapolate(g_prev, g_last, out, k: int, d: int):
     _check(load().hero_extrapolate(_ptr(g_prev), _ptr(g_last), _ptr(out), g_last.numel(), k, d,
                                    dtype_code(g_last.dtype), _stream()), "hero_extrapolate")
     return out
+
+
+# ---- diagnostics (Sec. 4.1) ------------------------------------------------------
+def hero_second_difference_moments(f_a, f_b, f_c, moments):
+    """moments (CUDA float64[2]) += (sum u, sum u^2) of u = f_a - 2 f_b + f_c."""
+    _require_cuda()
+    assert moments.is_cuda and moments.dtype == torch.float64 and moments.numel() == 2
+    _check(load().hero_second_difference_moments(_ptr(f_a), _ptr(f_b), _ptr(f_c), f_b.numel(), dtype_code(f_b.dtype),
+                                                 _ptr(moments), _stream()), "hero_second_difference_moments")
+    return moments
+
+
+def hero_extrapolation_error(g_prev, g_last, g_true, k: int, d: int, err):
+    """err (CUDA float64[2]) += (sum (Eq. 5 prediction - g_true)^2, sum g_true^2)."""
+    _require_cuda()
+    assert err.is_cuda and err.dtype == torch.float64 and err.numel() == 2
+    _check(load().hero_extrapolation_error(_ptr(g_prev), _ptr(g_last), _ptr(g_true), g_last.numel(), k, d,
+                                           dtype_code(g_last.dtype), _ptr(err), _stream()), "hero_extrapolation_error")
+    return err
 
 
 def hero_gather_rows(src, idx, dst):

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhero.so")
-SOURCES = ["hero_ctx.cu", "select.cu", "stream_kernels.cu", "simt_kernels.cu", "tc_gemm.cu", "tc_attention.cu", "qk_prep.cu"]
+SOURCES = ["hero_ctx.cu", "select.cu", "stream_kernels.cu", "simt_kernels.cu", "tc_gemm.cu", "tc_attention.cu", "qk_prep.cu", "diagnostics.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-Wno-deprecated-gpu-targets",
