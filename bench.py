@@ -325,10 +325,14 @@ def run_hero(args, cfg, rank, world, local_rank):
                              "frac": fl["gemm"] / (gemm_ms_blk * 1e-3) / 1e12 / peak,
                              "flops_per_block": fl["gemm"], "ms_per_block": gemm_ms_blk}}
         if breakdown["extrapolate"]["launches_per_step"]:
-            ext_ms = prof["extrapolate"][0] / prof["extrapolate"][1]
-            gbs = 6 * B * N * D * 2 / (ext_ms * 1e-3) / 1e9      # 5 reads + 1 write of [B,N,D] bf16
+            # all deep blocks in one pass per launch: four history tensors read per block, x read and written
+            # once per launch
+            n_deep = cfg["n_blocks"] - cfg["n_shallow"]
+            ext_ms = prof["extrapolate"][0] / n_prof
+            ext_bytes = B * N * D * 2 * (4 * n_deep + 2 * breakdown["extrapolate"]["launches_per_step"])
+            gbs = ext_bytes / (ext_ms * 1e-3) / 1e9
             roofline["extrapolate"] = {"achieved": gbs, "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
-                                       "ms_per_launch": ext_ms}
+                                       "ms_per_step": ext_ms, "bytes_per_step": ext_bytes, "blocks": n_deep}
 
     # end to end through the host entry point: pinned host buffers, H2D + step + D2H per call
     h_x = x.detach().cpu().pin_memory()

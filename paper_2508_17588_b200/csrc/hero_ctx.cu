@@ -291,6 +291,27 @@ int extrapolate_block(hero_ctx* c, int block, void* d_x, int k, int d) {
   return HERO_OK;
 }
 
+// Blocks [l0, l1) (all extrapolated) over elements [first, first + n) of the residual stream, at most
+// kMaxDeepGroup blocks per launch.
+int extrapolate_blocks(hero_ctx* c, int l0, int l1, void* d_x, long long first, long long n, int k, int d) {
+  for (int l = l0; l < l1; l += kMaxDeepGroup) {
+    DeepGroup grp;
+    grp.n_entries = 0;
+    for (int b = l; b < l1 && b < l + kMaxDeepGroup; ++b) {
+      const BlockMem& bm = c->blk[b];
+      if (bm.n_hist == 0) return HERO_ERR_STATE;
+      const int last = bm.last_slot, prev = bm.n_hist >= 2 ? (last ^ 1) : last;   // one slot only: Delta = 0
+      for (int br = 0; br < 2; ++br) {
+        grp.prev[grp.n_entries] = bm.hist[br][prev];
+        grp.last[grp.n_entries] = bm.hist[br][last];
+        grp.n_entries++;
+      }
+    }
+    HERO_LAUNCH(c, HERO_PROF_EXTRAPOLATE, launch_extrapolate_group(d_x, grp, first, n, k, d, c->cfg.dtype, c->stream));
+  }
+  return HERO_OK;
+}
+
 int validate(const hero_config* g) {
   if (g->n_blocks <= 0 || g->n_shallow < 0 || g->n_shallow > g->n_blocks) return HERO_ERR_ARG;
   if (g->hidden <= 0 || g->n_heads <= 0 || g->head_dim <= 0 || g->hidden != g->n_heads * g->head_dim) return HERO_ERR_ARG;
@@ -608,7 +629,8 @@ int hero_step(hero_ctx* c, int step, void* d_x, const void* d_temb) {
       HERO_TRY(extrapolate_stack(c, d_x, k, d));   // Eq. 5 once, on the sums over all deep blocks
       break;
     } else {
-      HERO_TRY(extrapolate_block(c, l, d_x, k, d));
+      HERO_TRY(extrapolate_blocks(c, l, g.n_blocks, d_x, 0, c->elems, k, d));   // the rest of the stack in one pass
+      break;
     }
   }
   return HERO_OK;

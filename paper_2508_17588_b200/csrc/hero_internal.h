@@ -78,6 +78,16 @@ int launch_extrapolate(const void* g_prev, const void* g_last, void* out, long l
 // x += e(attn history) ; x += e(ffn history)
 int launch_extrapolate_residual(void* x, const void* ga_prev, const void* ga_last, const void* gf_prev,
                                 const void* gf_last, long long n, int k, int d, int dtype, cudaStream_t s);
+// Several extrapolated blocks in one pass: x += sum over the group's (block, branch) entries of Eq. 5,
+// added in the order of the entries, for elements [first, first + n) of every tensor.
+constexpr int kMaxDeepGroup = 32;           // blocks per launch (two entries each)
+struct DeepGroup {
+  int n_entries;
+  const void* prev[2 * kMaxDeepGroup];
+  const void* last[2 * kMaxDeepGroup];
+};
+int launch_extrapolate_group(void* x, const DeepGroup& grp, long long first, long long n, int k, int d, int dtype,
+                             cudaStream_t s);
 // x = (x + ga) + gf
 int launch_residual2(void* x, const void* ga, const void* gf, long long n, int dtype, cudaStream_t s);
 // deep-stack collapse: x = (x + ga) + gf, acc += ga + gf (fp32);  x += s_last + (s_last - s_prev) * k/d
