@@ -34,6 +34,9 @@ struct BlockMem {
 
 using namespace hero;
 
+constexpr int kHostPieces = 4;                 // pieces of x copied back while the next one is computed
+constexpr long long kHostPieceAlign = 4096;    // elements; keeps every piece 16-byte aligned in both dtypes
+
 struct hero_ctx {
   hero_config cfg;
   cudaStream_t stream = nullptr;
@@ -51,6 +54,9 @@ struct hero_ctx {
   void* kv_cmp[2] = {nullptr, nullptr};
   int* att_list = nullptr;
   // rope 1: (cos, sin) of every (axis position, rotary pair), computed on the host in double precision
+  // hero_step_host: device-to-host copies of finished pieces of x run on this stream, behind the events
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t piece_done[kHostPieces] = {};
   float2* rope_tab = nullptr;
   int rope_pairs[3] = {0, 0, 0};
   void *ws_a = nullptr, *ws_q = nullptr, *ws_o = nullptr, *ws_u = nullptr;
@@ -363,6 +369,8 @@ const char* hero_last_cuda_error(void) { return g_last_error.c_str(); }
 void hero_destroy(hero_ctx* c) {
   if (!c) return;
   if (c->stream) cudaStreamSynchronize(c->stream); else cudaDeviceSynchronize();
+  if (c->copy_stream) { cudaStreamSynchronize(c->copy_stream); cudaStreamDestroy(c->copy_stream); }
+  for (cudaEvent_t e : c->piece_done) if (e) cudaEventDestroy(e);
   for (void* p : c->allocs) cudaFree(p);
   for (auto& sp : c->spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
   for (auto& sp : c->span_pool) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
@@ -580,7 +588,16 @@ int hero_is_full_step(const hero_ctx* c, int step) {
   return is_full(c->cfg, step) ? 1 : 0;
 }
 
+// One step of Algorithm 1.  With h_out set (hero_step_host) the deep blocks of a cached step run piece by
+// piece over x, and each finished piece is copied to h_out on the copy stream while the next one is
+// computed; *copied_out then tells the caller that nothing is left to copy.
+static int step_impl(hero_ctx* c, int step, void* d_x, const void* d_temb, void* h_out, bool* copied_out);
+
 int hero_step(hero_ctx* c, int step, void* d_x, const void* d_temb) {
+  return step_impl(c, step, d_x, d_temb, nullptr, nullptr);
+}
+
+static int step_impl(hero_ctx* c, int step, void* d_x, const void* d_temb, void* h_out, bool* copied_out) {
   if (!c || !d_x || !d_temb || step < 0) return HERO_ERR_ARG;
   if (!aligned16(d_x) || !aligned16(d_temb)) return HERO_ERR_ALIGN;
   const hero_config& g = c->cfg;
@@ -628,6 +645,23 @@ int hero_step(hero_ctx* c, int step, void* d_x, const void* d_temb) {
     } else if (collapse) {
       HERO_TRY(extrapolate_stack(c, d_x, k, d));   // Eq. 5 once, on the sums over all deep blocks
       break;
+    } else if (h_out && c->copy_stream && c->elems >= (long long)kHostPieces * kHostPieceAlign) {
+      // the rest of the stack, piece by piece, each piece on its way to the host as soon as it is final
+      const long long per = ((c->elems + kHostPieces - 1) / kHostPieces + kHostPieceAlign - 1) / kHostPieceAlign *
+                            kHostPieceAlign;
+      for (int p = 0; p < kHostPieces; ++p) {
+        const long long first = (long long)p * per;
+        const long long n = first >= c->elems ? 0 : (c->elems - first < per ? c->elems - first : per);
+        if (n <= 0) break;
+        HERO_TRY(extrapolate_blocks(c, l, g.n_blocks, d_x, first, n, k, d));
+        HERO_CUDA_TRY(cudaEventRecord(c->piece_done[p], c->stream));
+        HERO_CUDA_TRY(cudaStreamWaitEvent(c->copy_stream, c->piece_done[p], 0));
+        HERO_CUDA_TRY(cudaMemcpyAsync(static_cast<char*>(h_out) + first * c->esz,
+                                      static_cast<const char*>(d_x) + first * c->esz, (size_t)n * c->esz,
+                                      cudaMemcpyDeviceToHost, c->copy_stream));
+      }
+      *copied_out = true;
+      break;
     } else {
       HERO_TRY(extrapolate_blocks(c, l, g.n_blocks, d_x, 0, c->elems, k, d));   // the rest of the stack in one pass
       break;
@@ -641,9 +675,19 @@ int hero_step_host(hero_ctx* c, int step, void* h_x, const void* h_temb) {
   const size_t xb = (size_t)c->elems * c->esz, tb = (size_t)c->cfg.batch * c->cfg.temb_dim * c->esz;
   HERO_CUDA_TRY(cudaMemcpyAsync(c->x_stage, h_x, xb, cudaMemcpyHostToDevice, c->stream));
   HERO_CUDA_TRY(cudaMemcpyAsync(c->temb_stage, h_temb, tb, cudaMemcpyHostToDevice, c->stream));
-  HERO_TRY(hero_step(c, step, c->x_stage, c->temb_stage));
-  HERO_CUDA_TRY(cudaMemcpyAsync(h_x, c->x_stage, xb, cudaMemcpyDeviceToHost, c->stream));
+  if (!c->copy_stream) {
+    HERO_CUDA_TRY(cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
+    for (cudaEvent_t& e : c->piece_done) HERO_CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+  }
+  bool copied = false;
+  const int rc = step_impl(c, step, c->x_stage, c->temb_stage, h_x, &copied);
+  if (rc != HERO_OK) {                       // leave no copy in flight behind an error
+    cudaStreamSynchronize(c->copy_stream);
+    return rc;
+  }
+  if (!copied) HERO_CUDA_TRY(cudaMemcpyAsync(h_x, c->x_stage, xb, cudaMemcpyDeviceToHost, c->stream));
   HERO_CUDA_TRY(cudaStreamSynchronize(c->stream));
+  HERO_CUDA_TRY(cudaStreamSynchronize(c->copy_stream));
   return HERO_OK;
 }
 

@@ -164,6 +164,25 @@ def test_bf16_small_model_steps_teacher_forced(gate, attend_mode, qk):
     hero.close()
 
 
+def test_bf16_host_entry_point_matches_device_entry_point():
+    """hero_step_host copies x back piece by piece behind the deep blocks of a cached step; the result must be
+    the device entry point's, bit for bit, on full and cached steps (the last piece is ragged here)."""
+    cfgd = dict(SMALL_BF16, n_blocks=4, n_shallow=2)
+    weights = [S.block_weights(cfgd, l) for l in range(cfgd["n_blocks"])]
+    _, hero_a, _ = make_pair(cfgd, weights)
+    _, hero_b, _ = make_pair(cfgd, weights)
+    x0 = to_dev(S.tokens(cfgd), "bf16")
+    for s in range(cfgd["steps"]):
+        temb = to_dev(S.temb(cfgd, s), "bf16")
+        xd = x0.clone()
+        hero_a.hero_step(s, xd, temb)
+        xh = x0.cpu().pin_memory()
+        hero_b.hero_step_host(s, xh, temb.cpu().pin_memory())
+        assert torch.equal(xd.cpu(), xh), s
+    hero_a.hero_check_status(); hero_b.hero_check_status()
+    hero_a.close(); hero_b.close()
+
+
 def test_bf16_refresh_keeps_unselected_rows_bit_identical():
     cfgd = dict(SMALL_BF16, n_blocks=1, n_shallow=1)
     _, hero, _ = make_pair(cfgd)
