@@ -167,7 +167,25 @@ int run_attention(hero_ctx* c, const void* q, const void* k, const void* v, void
 }
 
 // Eq. 2 on the listed rows + Eq. 3's merge + the residual adds of Algorithm 1.
-int refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, const int* d_idx, int n_sel) {
+// adaLN vectors of blocks [l0, l1) into their slots of c->mod, at most kMaxModBatch blocks per launch
+int modulation_for_blocks(hero_ctx* c, int l0, int l1, const void* d_temb) {
+  const hero_config& g = c->cfg;
+  const int mod_ld = c->n_mod * g.hidden;
+  for (int l = l0; l < l1; l += kMaxModBatch) {
+    ModBatch mb;
+    mb.n = 0;
+    for (int b = l; b < l1 && b < l + kMaxModBatch; ++b, ++mb.n) {
+      mb.w_mod[mb.n] = c->w[b].w_mod; mb.b_mod[mb.n] = c->w[b].b_mod;
+      mb.mod[mb.n] = c->mod + (size_t)b * g.batch * mod_ld;
+    }
+    HERO_LAUNCH(c, HERO_PROF_MODULATION,
+                launch_modulation_batch(d_temb, mb, g.batch, mod_ld, g.temb_dim, g.dtype, c->stream));
+  }
+  return HERO_OK;
+}
+
+int refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, const int* d_idx, int n_sel,
+                  bool mod_ready = false) {
   const hero_config& g = c->cfg;
   const int B = g.batch, N = c->N, D = g.hidden, F = g.ffn_dim;
   const bool full = d_idx == nullptr;
@@ -191,14 +209,16 @@ int refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, const i
     kdst = bm.k; vdst = bm.v; ga = bm.g[0]; gf = bm.g[1];
   }
 
-  HERO_LAUNCH(c, HERO_PROF_MODULATION,
-              launch_modulation(d_temb, w.w_mod, w.b_mod, c->mod, B, mod_ld, g.temb_dim, g.dtype, c->stream));
-  const float* shift1 = c->mod;
-  const float* scale1 = c->mod + D;
-  const float* shift2 = c->mod + 2 * D;
-  const float* scale2 = c->mod + 3 * D;
-  const float* gate1 = g.has_gate ? c->mod + 4 * D : nullptr;
-  const float* gate2 = g.has_gate ? c->mod + 5 * D : nullptr;
+  float* mod = c->mod + (size_t)block * B * mod_ld;       // this block's slot; hero_step fills all slots up front
+  if (!mod_ready)
+    HERO_LAUNCH(c, HERO_PROF_MODULATION,
+                launch_modulation(d_temb, w.w_mod, w.b_mod, mod, B, mod_ld, g.temb_dim, g.dtype, c->stream));
+  const float* shift1 = mod;
+  const float* scale1 = mod + D;
+  const float* shift2 = mod + 2 * D;
+  const float* scale2 = mod + 3 * D;
+  const float* gate1 = g.has_gate ? mod + 4 * D : nullptr;
+  const float* gate2 = g.has_gate ? mod + 5 * D : nullptr;
 
   // attention branch
   HERO_LAUNCH(c, HERO_PROF_GATHER_LN,
@@ -448,7 +468,7 @@ int hero_init(hero_ctx** out, const hero_config* cfg, const hero_block_weights* 
   }
   A(&c->ws_a, tensor); A(&c->ws_q, tensor); A(&c->ws_o, tensor);
   A(&c->ws_u, (size_t)cfg->batch * c->N * cfg->ffn_dim * c->esz);
-  A((void**)&c->mod, (size_t)cfg->batch * c->n_mod * cfg->hidden * sizeof(float));
+  A((void**)&c->mod, (size_t)cfg->n_blocks * cfg->batch * c->n_mod * cfg->hidden * sizeof(float));
   A((void**)&c->idx_ws, (size_t)(cfg->n_shallow > 0 ? cfg->n_shallow : 1) * c->idx_cap * sizeof(int));
   A((void**)&c->d_status, 16);
   A(&c->x_stage, tensor);
@@ -607,7 +627,8 @@ static int step_impl(hero_ctx* c, int step, void* d_x, const void* d_temb, void*
       c->stack_new = c->stack_n == 0 ? 0 : (c->stack_last ^ 1);
       HERO_CUDA_TRY(cudaMemsetAsync(c->stack_hist[c->stack_new], 0, (size_t)c->elems * sizeof(float), c->stream));
     }
-    for (int l = 0; l < g.n_blocks; ++l) HERO_TRY(refresh_block(c, l, d_x, d_temb, nullptr, c->N));
+    HERO_TRY(modulation_for_blocks(c, 0, g.n_blocks, d_temb));
+    for (int l = 0; l < g.n_blocks; ++l) HERO_TRY(refresh_block(c, l, d_x, d_temb, nullptr, c->N, true));
     if (collapse) { c->stack_last = c->stack_new; if (c->stack_n < 2) c->stack_n++; }
     c->s_prev = c->s_last; c->s_last = step; c->n_full++;
     return HERO_OK;
@@ -634,10 +655,12 @@ static int step_impl(hero_ctx* c, int step, void* d_x, const void* d_temb, void*
     for (int l = 0; l < n_draws; ++l) { c->blk[l].ages_cur ^= 1; c->blk[l].calls++; }
     for (int l = n_draws; l < g.n_shallow; ++l) n_sel[l] = n_sel[0];
   }
+  HERO_TRY(modulation_for_blocks(c, 0, g.n_shallow, d_temb));
   for (int l = 0; l < g.n_blocks; ++l) {
     if (l < g.n_shallow) {
       if (n_sel[l] > 0) {
-        HERO_TRY(refresh_block(c, l, d_x, d_temb, c->idx_ws + (size_t)(g.share_selection ? 0 : l) * c->idx_cap, n_sel[l]));
+        HERO_TRY(refresh_block(c, l, d_x, d_temb, c->idx_ws + (size_t)(g.share_selection ? 0 : l) * c->idx_cap, n_sel[l],
+                               true));
       } else {
         HERO_LAUNCH(c, HERO_PROF_RESIDUAL,
                     launch_residual2(d_x, c->blk[l].g[0], c->blk[l].g[1], c->elems, g.dtype, c->stream));

@@ -114,6 +114,15 @@ int launch_gather_rows(const void* src, const int* idx, void* dst, int B, int N,
 int launch_scatter_rows(const void* src, const int* idx, void* dst, int B, int N, int n_sel, int D,
                         int dtype, cudaStream_t s);
 // mod[b, j] = b_mod[j] + sum_e silu(temb[b,e]) * w_mod[j,e]   (fp32 output)
+// The adaLN vectors of several blocks in one launch (they depend on the timestep embedding only).
+constexpr int kMaxModBatch = 64;
+struct ModBatch {
+  int n;
+  const void* w_mod[kMaxModBatch];
+  const void* b_mod[kMaxModBatch];
+  float* mod[kMaxModBatch];
+};
+int launch_modulation_batch(const void* temb, const ModBatch& batch, int B, int n_out, int E, int dtype, cudaStream_t s);
 int launch_modulation(const void* temb, const void* w_mod, const void* b_mod, float* mod, int B,
                       int n_out, int E, int dtype, cudaStream_t s);
 // a[m,:] = LN(x[row(m),:] (+ add[row(m),:])) * (1 + scale[b,:]) + shift[b,:]

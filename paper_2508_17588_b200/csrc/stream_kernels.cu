@@ -401,6 +401,51 @@ __global__ void __launch_bounds__(256) modulation_kernel(const T* __restrict__ t
   }
 }
 
+// The same for several blocks at once: blockIdx.y picks the block's weights and output.
+template <typename T>
+__global__ void __launch_bounds__(256) modulation_batch_kernel(const T* __restrict__ temb, const ModBatch batch, int B,
+                                                               int n_out, int E) {
+  extern __shared__ float s_act[];   // [B, E] silu(temb)
+  for (int i = threadIdx.x; i < B * E; i += blockDim.x) {
+    const float t = to_f(temb[i]);
+    s_act[i] = t / (1.0f + expf(-t));
+  }
+  __syncthreads();
+  const T* __restrict__ w_mod = static_cast<const T*>(batch.w_mod[blockIdx.y]);
+  const T* __restrict__ b_mod = static_cast<const T*>(batch.b_mod[blockIdx.y]);
+  float* __restrict__ mod = batch.mod[blockIdx.y];
+  const int lane = threadIdx.x & 31;
+  const int warps_per_block = blockDim.x >> 5;
+  using V = Vec<T>;
+  for (int j = blockIdx.x * warps_per_block + (threadIdx.x >> 5); j < n_out; j += gridDim.x * warps_per_block) {
+    float acc[kModMaxB];
+#pragma unroll
+    for (int b = 0; b < kModMaxB; ++b) acc[b] = 0.f;
+    const V* wrow = reinterpret_cast<const V*>(w_mod + (long long)j * E);
+    for (int c = lane; c < E / V::N; c += 32) {
+      float wf[V::N];
+      V wv; wv.raw = __ldg(&wrow[c].raw);
+      wv.unpack(wf);
+#pragma unroll
+      for (int b = 0; b < kModMaxB; ++b) {
+        if (b < B) {
+#pragma unroll
+          for (int q = 0; q < V::N; ++q) acc[b] = fmaf(s_act[b * E + c * V::N + q], wf[q], acc[b]);
+        }
+      }
+    }
+#pragma unroll
+    for (int b = 0; b < kModMaxB; ++b) {
+      if (b < B) {
+        float v = acc[b];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+        if (lane == 0) mod[(long long)b * n_out + j] = v + to_f(b_mod[j]);
+      }
+    }
+  }
+}
+
 // ------------------------------------------------------------------ gather + LayerNorm + modulate (Eq. 2 prologue)
 // One CTA per refreshed row: the row (plus, for the FFN branch, the not-yet-added attention
 // output of the same row) is read once into shared memory as fp32, mean and biased variance
@@ -681,6 +726,26 @@ int launch_gather_rows(const void* src, const int* idx, void* dst, int B, int N,
 int launch_scatter_rows(const void* src, const int* idx, void* dst, int B, int N, int n_sel, int D, int dtype,
                         cudaStream_t s) {
   return move_rows(false, src, idx, dst, B, N, n_sel, D, dtype, s);
+}
+
+int launch_modulation_batch(const void* temb, const ModBatch& batch, int B, int n_out, int E, int dtype,
+                            cudaStream_t s) {
+  if (B > kModMaxB || batch.n < 0 || batch.n > kMaxModBatch) return HERO_ERR_ARG;
+  if (batch.n == 0) return HERO_OK;
+  const size_t smem = (size_t)B * E * sizeof(float);
+  int bx = (n_out + 7) / 8;
+  const int cap = (num_sms() * 8 + batch.n - 1) / batch.n;     // about eight CTAs per SM over the whole grid
+  if (bx > cap) bx = cap < 1 ? 1 : cap;
+  const dim3 grid(bx, batch.n);
+  if (dtype == HERO_DTYPE_BF16) {
+    if (E % 8) return HERO_ERR_ALIGN;
+    modulation_batch_kernel<__nv_bfloat16><<<grid, 256, smem, s>>>((const __nv_bfloat16*)temb, batch, B, n_out, E);
+  } else {
+    if (E % 4) return HERO_ERR_ALIGN;
+    modulation_batch_kernel<float><<<grid, 256, smem, s>>>((const float*)temb, batch, B, n_out, E);
+  }
+  HERO_CUDA_TRY(cudaGetLastError());
+  return HERO_OK;
 }
 
 int launch_modulation(const void* temb, const void* w_mod, const void* b_mod, float* mod, int B, int n_out, int E,
