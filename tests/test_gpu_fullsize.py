@@ -25,6 +25,7 @@ def H():
 CASES = {
     "cogvideox_block_25": dict(S.CONFIGS["block"], ratio_num=1, ratio_den=4),
     "cogvideox_block_25_qk_norm_rope": dict(S.CONFIGS["block"], ratio_num=1, ratio_den=4, qk_norm=1, rope=1),
+    "cogvideox_block_25_attend_refreshed": dict(S.CONFIGS["block"], ratio_num=1, ratio_den=4, attend_mode=1),
     "aether_block_10": dict(S.CONFIGS["aether"], n_blocks=1, n_shallow=1, ratio_num=1, ratio_den=10, full_interval=0),
 }
 
