@@ -426,6 +426,16 @@ def run_hero(args, cfg, rank, world, local_rank):
         if base_qk:
             line["qk_norm_rope_variant"] = base_qk
         if roofline:
+            # the same launch against the exponential unit: one ex2 per score, 16 per clock per SM (measured on
+            # this chip), at the SM clock sampled during the timed region
+            if clocks.get("sm_mhz") and cfg["head_dim"] == 64:
+                sms = torch.cuda.get_device_properties(device).multi_processor_count
+                exps = roofline["flops_per_launch"] / (4.0 * cfg["head_dim"])      # 4 * head_dim flop per score
+                peak_exp = 16.0 * sms * clocks["sm_mhz"] * 1e6
+                ach_exp = exps / (roofline["ms_per_launch"] * 1e-3)
+                roofline["exp_unit"] = {"achieved": ach_exp / 1e12, "peak": peak_exp / 1e12, "unit": "Texp/s",
+                                        "frac": ach_exp / peak_exp,
+                                        "note": "secondary bound of the attention kernel at head_dim 64"}
             line["roofline"] = roofline
         if cpu_baseline:
             line["cpu_baseline"] = cpu_baseline
