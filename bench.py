@@ -577,6 +577,24 @@ def run_kernels(args):
         hero.hero_check_status()
         hero.close()
         del weights, x
+    if want("deep_group") and not args.small:
+        # a stack of four extrapolated blocks and nothing else: its cached step is exactly one launch of the
+        # grouped pass (16 history tensors read, x read and written once: 36 B per element)
+        gcfg = dict(S.CONFIGS["block"], n_blocks=4, n_shallow=0)
+        weights = build_device_weights(gcfg, dev)
+        hero = H.Hero(gcfg, weights)
+        x = S.device_normal(gcfg["seed"], "x0", (B, N, D), 1.0, 0, None, dev).to(bf)
+        temb = S.device_normal(gcfg["seed"], "temb", (B, gcfg["temb_dim"]), 1.0, 0, None, dev).to(bf)
+        for s_ in range(2):
+            hero.hero_step(s_, x, temb)
+        state = {"s": 2}
+
+        def one_group():
+            hero.hero_step(state["s"], x, temb); state["s"] += 1
+        hbm("extrapolate_group_4_blocks", _time_flushed(one_group, iters, warm, flush), (8 * 4 + 4) * B * N * D)
+        hero.hero_check_status()
+        hero.close()
+        del weights, x
     if want("block") and not args.small:
         bcfg = dict(S.CONFIGS["block"])
         weights = build_device_weights(bcfg, dev)
@@ -613,7 +631,7 @@ def main():
     ap.add_argument("--impl", default="hero", choices=["hero", "reference"])
     ap.add_argument("--workload", default="dit42", choices=["dit42", "aether", "paper_hp", "tiny", "kernels"])
     ap.add_argument("--only", default="", help="kernels workload: comma list of select,extrapolate,gather,scatter,"
-                                               "attention,gemm,deep,block,diagnostics")
+                                               "attention,gemm,deep,deep_group,block,diagnostics")
     ap.add_argument("--small", action="store_true", help="kernels workload: profiler-sized tensor-core cases")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-collapse", action="store_true", help="skip the variant runs (collapsed deep stack, refreshed-rows-only attention)")
