@@ -22,7 +22,11 @@
  *     temb_dim must be multiples of 8 and head_dim must be 64.
  *   - All work is enqueued on the CUDA stream given to hero_init; no call
  *     synchronises the device unless stated.  Calls on one context must not
- *     overlap in time.
+ *     overlap in time.  hero_step, hero_refresh_block and the extrapolation calls
+ *     only enqueue kernels (no allocation, no host read), so they may be recorded
+ *     by a stream capture into a CUDA graph; the context's host-side counters
+ *     advance at capture time, once, as if the step had run, so each captured step
+ *     is to be replayed exactly once.
  *   - Return value: HERO_OK (0) or a negative HERO_ERR_* code.  After an argument
  *     error nothing has been launched.  No exception crosses this boundary.
  */
