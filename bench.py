@@ -11,7 +11,9 @@ in `config` together with the 50-step schedule average.
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl hero|reference] [--workload dit42|aether|paper_hp|tiny|kernels [--only LIST] [--small]]
 
 Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank runs its own sequence on its
-own GPU (independent problems, no data-path collective): "scaling": "weak".
+own GPU (independent problems, no data-path collective): "scaling": "weak".  `--cfg-split` instead
+gives each rank batch/N items of one problem (the guidance pair, one item per GPU at N = 2; the ranks draw
+the same selection lists on their own, nothing is exchanged): "scaling": "strong".
 """
 from __future__ import annotations
 
@@ -212,6 +214,16 @@ def whole_job_throughput(tokens_per_rank_step: int, world: int, ms_per_step: flo
     return world * tokens_per_rank_step / (ms_per_step * 1e-3)
 
 
+def shard_cfg_pair(cfg: dict, rank: int, world: int):
+    """The items of one problem's batch (the classifier-free-guidance pair) split over the ranks: every rank
+    keeps the seed, hence the same selection lists, and runs batch/world sequences; nothing is exchanged.
+    Returns the rank's config and its slice of the batch axis."""
+    if world < 1 or not 0 <= rank < world or cfg["batch"] % world:
+        raise ValueError(f"batch {cfg['batch']} does not split over {world} ranks")
+    per = cfg["batch"] // world
+    return dict(cfg, batch=per), slice(rank * per, (rank + 1) * per)
+
+
 def rank_seed(base_seed: int, rank: int) -> int:
     """Each rank draws its own problem."""
     return base_seed + rank
@@ -245,13 +257,19 @@ def run_hero(args, cfg, rank, world, local_rank):
         dist.init_process_group("nccl", device_id=device)
     dt = torch.bfloat16 if cfg["dtype"] == "bf16" else torch.float32
     run_cfg = dict(cfg, full_interval=0)         # after the two warm-up full steps every step is cached
-    run_cfg["seed"] = rank_seed(cfg["seed"], rank)   # each rank its own sequence (independent problems)
+    B_all, N, D = cfg["batch"], S.n_rows(cfg), cfg["hidden"]
+    if args.cfg_split:
+        # one problem, its batch items split over the ranks (strong scaling, no exchange)
+        run_cfg, part = shard_cfg_pair(run_cfg, rank, world)
+    else:
+        run_cfg["seed"] = rank_seed(cfg["seed"], rank)   # each rank its own sequence (independent problems)
+        part = slice(0, B_all)
     weights = build_device_weights(run_cfg, device)
     hero = H.Hero(run_cfg, weights)
-    B, N, D = cfg["batch"], S.n_rows(cfg), cfg["hidden"]
+    B = run_cfg["batch"]
     tokens = B * N
-    x = S.device_normal(run_cfg["seed"], "x0", (B, N, D), 1.0, 0, None, device).to(dt)
-    tembs = [S.device_normal(run_cfg["seed"], "temb", (B, cfg["temb_dim"]), 1.0, s, None, device).to(dt)
+    x = S.device_normal(run_cfg["seed"], "x0", (B_all, N, D), 1.0, 0, None, device).to(dt)[part].contiguous()
+    tembs = [S.device_normal(run_cfg["seed"], "temb", (B_all, cfg["temb_dim"]), 1.0, s, None, device).to(dt)[part].contiguous()
              for s in range(8)]
 
     def ev():
@@ -307,7 +325,7 @@ def run_hero(args, cfg, rank, world, local_rank):
     roofline = None
     if cfg["n_shallow"] and prof["attention"][1]:
         n_sel = statistics.mean(n_sel_seen)
-        fl = refresh_flops(cfg, n_sel)
+        fl = refresh_flops(run_cfg, n_sel)
         att_ms = prof["attention"][0] / prof["attention"][1]
         gemm_ms_blk = prof["gemm"][0] / prof["attention"][1]          # four GEMMs per attention launch
         achieved = fl["attention"] / (att_ms * 1e-3) / 1e12
@@ -411,13 +429,15 @@ def run_hero(args, cfg, rank, world, local_rank):
                      (cfg["full_interval"] > 0 and (s - (cfg["warmup_full_steps"] - 1)) % cfg["full_interval"] == 0))
         sched_ms = (n_full * full_ms + (cfg["steps"] - n_full) * ms_per_step) / cfg["steps"]
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "strong" if args.cfg_split and world > 1 else "weak",
                 "vs_baseline": None, "dtype": cfg["dtype"], "data": "synthetic",
                 "config": dict(workload_config(args, cfg),
                                l2="inputs larger than L2 (each step streams > 30 GB of caches)",
                                full_step_ms=full_ms, schedule_avg_ms_per_step=sched_ms,
                                schedule="%d full + %d cached of %d steps" % (n_full, cfg["steps"] - n_full, cfg["steps"]),
-                               device_bytes=mem, parallelism="replicas" if world > 1 else "single"),
+                               device_bytes=mem,
+                               parallelism=("cfg_split" if args.cfg_split else "replicas") if world > 1 else "single"),
                 "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "breakdown_ms": breakdown}
         if collapsed:
             line["deep_collapse_variant"] = collapsed
@@ -634,6 +654,8 @@ def main():
                                                "attention,gemm,deep,deep_group,block,diagnostics")
     ap.add_argument("--small", action="store_true", help="kernels workload: profiler-sized tensor-core cases")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cfg-split", action="store_true",
+                    help="with --gpus N: split the batch items of ONE problem over the ranks instead of running N problems")
     ap.add_argument("--no-collapse", action="store_true", help="skip the variant runs (collapsed deep stack, refreshed-rows-only attention)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))

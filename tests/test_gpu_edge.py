@@ -123,6 +123,37 @@ def test_cached_step_can_be_captured_in_a_cuda_graph(dtype):
         plain.close(); graphed.close()
 
 
+@pytest.mark.parametrize("name", ["tiny_fp32", "small_bf16"])
+def test_batch_items_in_separate_contexts_reproduce_the_joint_batch(name):
+    """The split of a problem's batch over GPUs (one item per rank, no exchange) emulated on one GPU: two
+    contexts of batch 1 run one after the other on the two items give the joint context's result bit for
+    bit, with the same selection lists."""
+    import bench
+    if name == "tiny_fp32":
+        cfgd = dict(S.CONFIGS["tiny"], batch=2, full_interval=3, steps=6)
+    else:
+        cfgd = dict(n_blocks=3, n_shallow=2, hidden=256, n_heads=4, head_dim=64, ffn_dim=768, temb_dim=64, batch=2,
+                    frames=3, grid_h=9, grid_w=11, n_text=10, patch_h=2, patch_w=2, ratio_num=1, ratio_den=4,
+                    quota_mode=0, warmup_full_steps=2, full_interval=3, dtype="bf16", has_gate=0, seed=23, steps=6)
+    dt = cfgd["dtype"]
+    weights = [S.block_weights(cfgd, l) for l in range(cfgd["n_blocks"])]
+    _, joint, _ = make_pair(cfgd, weights)
+    parts = [bench.shard_cfg_pair(cfgd, r, 2) for r in range(2)]
+    ranks = [make_pair(c, weights)[1] for c, _ in parts]
+    x_host = S.tokens(cfgd)
+    for s in range(cfgd["steps"]):
+        temb = S.temb(cfgd, s)
+        x = to_dev(x_host, dt)
+        joint.hero_step(s, x, to_dev(temb, dt))
+        for (c, sl), h in zip(parts, ranks):
+            y = to_dev(x_host[sl], dt)
+            h.hero_step(s, y, to_dev(temb[sl], dt))
+            assert torch.equal(y, x[sl]), (s, sl)
+            assert torch.equal(h.hero_state_get(0, "ages"), joint.hero_state_get(0, "ages"))
+    for h in ranks + [joint]:
+        h.hero_check_status(); h.close()
+
+
 def test_call_order_and_argument_errors_with_a_live_context():
     h = H()
     cfgd = dict(S.CONFIGS["tiny"])
