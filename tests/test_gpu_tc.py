@@ -201,3 +201,31 @@ def test_bf16_refresh_keeps_unselected_rows_bit_identical():
         assert torch.equal(after[:, keep], b4[:, keep]), name
         assert not torch.equal(after[:, rows], b4[:, rows]), name
     hero.close()
+
+
+def test_free_running_drift_over_the_42_block_50_step_schedule_in_miniature(capsys):
+    """No teacher forcing: a 42-block model (14 refresh + 28 extrapolated, full step every 5, 50 steps) at
+    a small width runs freely on both sides, bf16 caches on the GPU against float64 in the oracle, and the
+    per-step distance of the outputs is reported.  Selection is integer work, so lists and ages stay
+    bit-identical however far the values drift.  Only a loose bound is asserted: the number is a report."""
+    cfgd = dict(SMALL_BF16, n_blocks=42, n_shallow=14, full_interval=5, steps=50, seed=31)
+    weights = [S.block_weights(cfgd, l) for l in range(cfgd["n_blocks"])]
+    orc, hero, _ = make_pair(cfgd, weights)
+    x_host = S.tokens(cfgd)
+    errs = []
+    for s in range(cfgd["steps"]):
+        temb = S.temb(cfgd, s)
+        want = orc.step(s, x_host, temb)
+        x = to_dev(x_host, "bf16")
+        hero.hero_step(s, x, to_dev(temb, "bf16"))
+        errs.append(rel_l2(to_host(x), want))
+        for l in (0, 13):
+            assert np.array_equal(hero.hero_state_get(l, "ages").numpy(), orc.blocks[l].ages), (s, l)
+    hero.hero_check_status()
+    hero.close()
+    full = [e for s, e in enumerate(errs) if orc.is_full_step(s)]
+    cached = [e for s, e in enumerate(errs) if not orc.is_full_step(s)]
+    with capsys.disabled():
+        print(f"\nfree-running drift, 42 blocks x 50 steps (bf16 vs float64): full steps max {max(full):.2e}, "
+              f"cached steps max {max(cached):.2e}, last step {errs[-1]:.2e}")
+    assert np.isfinite(errs).all() and max(errs) <= 5e-2
