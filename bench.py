@@ -499,7 +499,7 @@ def run_kernels(args):
     only = set(args.only.split(",")) if args.only else None
     want = lambda name: only is None or name in only
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-    iters, warm = max(args.steps, 5), max(args.warmup, 3)
+    iters, warm = max(args.steps, 5), max(args.warmup, 3)        # default 20 calls per kernel, median
     bf = torch.bfloat16
     out = {}
 
@@ -646,7 +646,8 @@ def run_kernels(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=None,
+                    help="timed steps (default 10; kernels workload: timed calls per kernel, default 20)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="hero", choices=["hero", "reference"])
     ap.add_argument("--workload", default="dit42", choices=["dit42", "aether", "paper_hp", "tiny", "kernels"])
@@ -658,6 +659,8 @@ def main():
                     help="with --gpus N: split the batch items of ONE problem over the ranks instead of running N problems")
     ap.add_argument("--no-collapse", action="store_true", help="skip the variant runs (collapsed deep stack, refreshed-rows-only attention)")
     args = ap.parse_args()
+    if args.steps is None:
+        args.steps = 20 if args.workload == "kernels" else 10
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
