@@ -53,14 +53,14 @@ struct hero_ctx {
   // attend_mode 1: compact K/V of the rows a cached step attends to (text + refreshed) and their list
   void* kv_cmp[2] = {nullptr, nullptr};
   int* att_list = nullptr;
-  // rope 1: (cos, sin) of every (axis position, rotary pair), computed on the host in double precision
   // hero_step_host: device-to-host copies of finished pieces of x run on this stream, behind the events
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t piece_done[kHostPieces] = {};
+  // rope 1: (cos, sin) of every (axis position, rotary pair), computed on the host in double precision
   float2* rope_tab = nullptr;
   int rope_pairs[3] = {0, 0, 0};
   void *ws_a = nullptr, *ws_q = nullptr, *ws_o = nullptr, *ws_u = nullptr;
-  float* mod = nullptr;                  // [B, n_mod*D] adaLN vectors of the current block
+  float* mod = nullptr;                  // [n_blocks, B, n_mod*D] adaLN vectors, one slot per block
   int* idx_ws = nullptr;                 // [n_shallow, idx_cap] selection lists of the current step
   int* d_status = nullptr;
   void *x_stage = nullptr, *temb_stage = nullptr;
@@ -166,7 +166,6 @@ int run_attention(hero_ctx* c, const void* q, const void* k, const void* v, void
   return launch_simt_attention(q, k, v, o, g.batch, n_q, c->N, g.n_heads, g.head_dim, g.dtype, c->stream);
 }
 
-// Eq. 2 on the listed rows + Eq. 3's merge + the residual adds of Algorithm 1.
 // adaLN vectors of blocks [l0, l1) into their slots of c->mod, at most kMaxModBatch blocks per launch
 int modulation_for_blocks(hero_ctx* c, int l0, int l1, const void* d_temb) {
   const hero_config& g = c->cfg;
@@ -184,6 +183,8 @@ int modulation_for_blocks(hero_ctx* c, int l0, int l1, const void* d_temb) {
   return HERO_OK;
 }
 
+// Eq. 2 on the listed rows + Eq. 3's merge + the residual adds of Algorithm 1.  mod_ready: the block's adaLN
+// vectors are in its slot already (hero_step computes them for all blocks of the step in one launch).
 int refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, const int* d_idx, int n_sel,
                   bool mod_ready = false) {
   const hero_config& g = c->cfg;
