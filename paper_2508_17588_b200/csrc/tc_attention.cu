@@ -193,10 +193,13 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const int h = (blockIdx.x / q_groups) % heads;
   const int b = blockIdx.x / (q_groups * heads);
   const int n_kv = (N + kKT - 1) / kKT;
+  // the last query group of a (batch, head) may reach into its second tile by no row at all: that tile's
+  // issuer and softmax warps then have nothing to do and the K/V stages are released by one issuer alone
+  const int n_tiles = (qg * kQTiles + 1) * kQT < n_q ? kQTiles : 1;
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
-    for (int i = 0; i < kKvStages; ++i) { mbar_init(&kv_full[i], 1); mbar_init(&kv_empty[i], kQTiles); }
+    for (int i = 0; i < kKvStages; ++i) { mbar_init(&kv_full[i], 1); mbar_init(&kv_empty[i], n_tiles); }
     for (int i = 0; i < 4; ++i) { mbar_init(&s_full[i], 1); mbar_init(&p_full[i], 4); }
     for (int i = 0; i < kQTiles; ++i) mbar_init(&pv_full[i], 1);
     *abort_flag = 0;
@@ -212,8 +215,8 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      mbar_expect_tx(q_full, kQTiles * kQBytes);
-      for (int t = 0; t < kQTiles; ++t)
+      mbar_expect_tx(q_full, n_tiles * kQBytes);
+      for (int t = 0; t < n_tiles; ++t)
         tma_load_2d(s_q + t * kQBytes, &tm_q, q_full, h * kHD, b * n_q + (qg * kQTiles + t) * kQT);
       int stage = 0; uint32_t phase = 0;
       for (int j = 0; j < n_kv; ++j) {
@@ -231,7 +234,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     }
   } else if (warp == 1 || warp == 2) {
     // ------------------------------------------------------------ MMA issuer of query tile t
-    if (lane == 0) {
+    if (lane == 0 && warp - 1 < n_tiles) {
       const int t = warp - 1;
       constexpr uint32_t idesc_s = idesc_bf16(kQT, kKT, 0);    // S = Q K^T : both operands K-contiguous
       constexpr uint32_t idesc_pv = idesc_bf16(kQT, kHD, 1);   // O += P V  : V is N(head_dim)-contiguous
@@ -269,7 +272,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
       }
     }
-  } else if (warp >= kFirstSoftmaxWarp) {
+  } else if (warp >= kFirstSoftmaxWarp && ((warp - kFirstSoftmaxWarp) >> 2) < n_tiles) {
     // ------------------------------------------------------------ softmax
     const int t = (warp - kFirstSoftmaxWarp) >> 2;     // query tile of this softmax group
     const int quad = warp & 3;                         // TMEM lane quadrant this warp may touch
