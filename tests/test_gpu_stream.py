@@ -158,3 +158,31 @@ def test_select_bit_exact(name):
         hero.hero_select_tokens(0, small)
     assert e.value.code == -3
     hero.close()
+
+
+@pytest.mark.parametrize("case", range(24))
+def test_select_bit_exact_on_random_geometries(case):
+    """A seeded sweep over grids, patch shapes (also larger than the grid, also 1x1), ratios, quota and
+    tracking modes, with and without text rows: lists, ages and counters bit for bit over 12 calls."""
+    rng = np.random.default_rng(1000 + case)
+    den = int(rng.integers(1, 12))
+    cfgd = dict(S.CONFIGS["tiny"], hidden=64, n_heads=1, head_dim=64, ffn_dim=64, temb_dim=8, n_blocks=1, n_shallow=1,
+                frames=int(rng.integers(1, 5)), grid_h=int(rng.integers(1, 14)), grid_w=int(rng.integers(1, 14)),
+                patch_h=int(rng.integers(1, 5)), patch_w=int(rng.integers(1, 5)), n_text=int(rng.integers(0, 6)),
+                ratio_num=int(rng.integers(1, den + 1)), ratio_den=den, quota_mode=int(rng.integers(0, 2)),
+                track_mode=int(rng.integers(0, 2)), seed=int(rng.integers(0, 2 ** 40)))
+    cfg = O.Config.from_dict(cfgd)
+    w = [{k: np.zeros(s, np.float32) for k, s in S.weight_shapes(cfgd).items()}]
+    h = H()
+    hero = h.Hero(cfgd, [h.device_weights(x, "fp32") for x in w])
+    ages = np.zeros(cfg.n_video, np.uint16)
+    for call in range(12):
+        want_rows, ages = O.select_tokens(cfg, ages, 0, call)
+        assert hero.hero_next_n_sel(0) == len(want_rows), (cfgd, call)
+        idx = torch.full((max(cfg.n_video, 1),), -1, dtype=torch.int32, device="cuda")
+        n = hero.hero_select_tokens(0, idx)
+        got = idx.cpu().numpy()
+        assert n == len(want_rows) and np.array_equal(got[:n], want_rows), (cfgd, call)
+        assert (got[n:] == -1).all()
+        assert np.array_equal(hero.hero_state_get(0, "ages").numpy(), ages), (cfgd, call)
+    hero.close()

@@ -57,7 +57,11 @@ def test_gemm_many_tiles_per_cta():
 
 # ---------------------------------------------------------------- attention
 @pytest.mark.parametrize("B,n_q,N,heads", [(1, 128, 128, 1), (1, 1, 1, 1), (2, 37, 200, 2), (1, 130, 513, 3),
-                                           (2, 300, 1000, 2), (1, 64, 2300, 1)])
+                                           (2, 300, 1000, 2), (1, 64, 2300, 1),
+                                           # query counts around the 128-row tile and 256-row group edges: the
+                                           # second tile of the last group is empty, one row full, or full
+                                           (1, 129, 300, 2), (2, 255, 193, 1), (1, 256, 97, 2), (1, 257, 300, 1),
+                                           (2, 384, 200, 1), (1, 385, 290, 2), (1, 640, 100, 1)])
 def test_attention_matches_oracle(B, n_q, N, heads):
     rng = np.random.default_rng(B * 7 + n_q + N)
     D = heads * 64
