@@ -363,10 +363,13 @@ template <typename T>
 __global__ void __launch_bounds__(256) modulation_kernel(const T* __restrict__ temb, const T* __restrict__ w_mod,
                                                          const T* __restrict__ b_mod, float* __restrict__ mod,
                                                          int B, int n_out, int E) {
-  extern __shared__ float s_act[];   // [B, E] silu(temb)
+  // silu(temb), laid out [B][V::N][E / V::N]: element e of a row sits at (e % V::N) * (E / V::N) + e / V::N, so
+  // that the lanes of a warp, which hold consecutive 16-byte packets of a weight row, read consecutive words
+  extern __shared__ float s_act[];
   for (int i = threadIdx.x; i < B * E; i += blockDim.x) {
     const float t = to_f(temb[i]);
-    s_act[i] = t / (1.0f + expf(-t));
+    const int b = i / E, e = i - b * E;
+    s_act[b * E + (e % Vec<T>::N) * (E / Vec<T>::N) + e / Vec<T>::N] = t / (1.0f + expf(-t));
   }
   __syncthreads();
   const int lane = threadIdx.x & 31;
@@ -385,7 +388,7 @@ __global__ void __launch_bounds__(256) modulation_kernel(const T* __restrict__ t
       for (int b = 0; b < kModMaxB; ++b) {
         if (b < B) {
 #pragma unroll
-          for (int q = 0; q < V::N; ++q) acc[b] = fmaf(s_act[b * E + c * V::N + q], wf[q], acc[b]);
+          for (int q = 0; q < V::N; ++q) acc[b] = fmaf(s_act[b * E + q * (E / V::N) + c], wf[q], acc[b]);
         }
       }
     }
@@ -405,10 +408,13 @@ __global__ void __launch_bounds__(256) modulation_kernel(const T* __restrict__ t
 template <typename T>
 __global__ void __launch_bounds__(256) modulation_batch_kernel(const T* __restrict__ temb, const ModBatch batch, int B,
                                                                int n_out, int E) {
-  extern __shared__ float s_act[];   // [B, E] silu(temb)
+  // silu(temb), laid out [B][V::N][E / V::N]: element e of a row sits at (e % V::N) * (E / V::N) + e / V::N, so
+  // that the lanes of a warp, which hold consecutive 16-byte packets of a weight row, read consecutive words
+  extern __shared__ float s_act[];
   for (int i = threadIdx.x; i < B * E; i += blockDim.x) {
     const float t = to_f(temb[i]);
-    s_act[i] = t / (1.0f + expf(-t));
+    const int b = i / E, e = i - b * E;
+    s_act[b * E + (e % Vec<T>::N) * (E / Vec<T>::N) + e / Vec<T>::N] = t / (1.0f + expf(-t));
   }
   __syncthreads();
   const T* __restrict__ w_mod = static_cast<const T*>(batch.w_mod[blockIdx.y]);
@@ -430,7 +436,7 @@ __global__ void __launch_bounds__(256) modulation_batch_kernel(const T* __restri
       for (int b = 0; b < kModMaxB; ++b) {
         if (b < B) {
 #pragma unroll
-          for (int q = 0; q < V::N; ++q) acc[b] = fmaf(s_act[b * E + c * V::N + q], wf[q], acc[b]);
+          for (int q = 0; q < V::N; ++q) acc[b] = fmaf(s_act[b * E + q * (E / V::N) + c], wf[q], acc[b]);
         }
       }
     }
@@ -734,7 +740,7 @@ int launch_modulation_batch(const void* temb, const ModBatch& batch, int B, int 
   if (batch.n == 0) return HERO_OK;
   const size_t smem = (size_t)B * E * sizeof(float);
   int bx = (n_out + 7) / 8;
-  const int cap = (num_sms() * 8 + batch.n - 1) / batch.n;     // about eight CTAs per SM over the whole grid
+  const int cap = num_sms() * 8 / batch.n;     // at most eight CTAs per SM over the whole grid: one wave, no tail
   if (bx > cap) bx = cap < 1 ? 1 : cap;
   const dim3 grid(bx, batch.n);
   if (dtype == HERO_DTYPE_BF16) {
