@@ -173,7 +173,11 @@ int hero_extrapolate_deep_stack(hero_ctx *ctx, void *d_x, int k, int d);
  * blocks and extrapolation in deep ones with k, d taken from the recorded full steps. */
 int hero_step(hero_ctx *ctx, int step, void *d_x, const void *d_temb);
 /* Same with HOST buffers: copies h_x and h_temb to the device, runs the step, copies x
- * back into h_x and synchronises the stream.  Pinned host memory overlaps best. */
+ * back into h_x and synchronises the stream.  With pinned (page-locked, device-visible) host buffers a cached
+ * step overlaps both copies with the work: the first refresh block normalises its rows straight out of h_x
+ * while x uploads on a second stream, and finished pieces of x travel back while the deep blocks run on the
+ * next piece.  Pageable buffers work too, without the overlap.  h_x must not be written by the caller during
+ * the call. */
 int hero_step_host(hero_ctx *ctx, int step, void *h_x, const void *h_temb);
 /* 1 if hero_step would run `step` as a full step. */
 int hero_is_full_step(const hero_ctx *ctx, int step);

@@ -56,6 +56,11 @@ struct hero_ctx {
   // hero_step_host: device-to-host copies of finished pieces of x run on this stream, behind the events
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t piece_done[kHostPieces] = {};
+  // hero_step_host, cached step with a pinned host buffer: the first refresh block normalises its rows
+  // straight out of host memory while the bulk upload of x is still under way on the copy stream
+  cudaEvent_t x_uploaded = nullptr;
+  const void* first_rows_src = nullptr;   // device alias of the caller's pinned x, consumed by one refresh_block
+  bool wait_x_upload = false;
   // rope 1: (cos, sin) of every (axis position, rotary pair), computed on the host in double precision
   float2* rope_tab = nullptr;
   int rope_pairs[3] = {0, 0, 0};
@@ -222,8 +227,10 @@ int refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, const i
   const float* gate2 = g.has_gate ? mod + 5 * D : nullptr;
 
   // attention branch
+  const void* x_rows = c->first_rows_src ? c->first_rows_src : d_x;
+  c->first_rows_src = nullptr;
   HERO_LAUNCH(c, HERO_PROF_GATHER_LN,
-              launch_gather_ln_modulate(d_x, nullptr, d_idx, shift1, scale1, mod_ld, c->ws_a, B, N, n_sel, D, 1e-5f,
+              launch_gather_ln_modulate(x_rows, nullptr, d_idx, shift1, scale1, mod_ld, c->ws_a, B, N, n_sel, D, 1e-5f,
                                         g.dtype, c->stream));
   GemmOut o_qkv = {};
   o_qkv.ptr[0] = c->ws_q; o_qkv.ld[0] = D; o_qkv.scatter[0] = 0;
@@ -266,6 +273,10 @@ int refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, const i
   o_attn.gate = gate1; o_attn.gate_ld = mod_ld;
   HERO_TRY(run_gemm(c, c->ws_o, w.w_o, w.b_o, M, D, D, o_attn));
 
+  if (c->wait_x_upload) {                  // from here on x is read from the device copy
+    c->wait_x_upload = false;
+    HERO_CUDA_TRY(cudaStreamWaitEvent(c->stream, c->x_uploaded, 0));
+  }
   // FFN branch: its input rows are x + G_attn (the residual add is applied to x once, below)
   HERO_LAUNCH(c, HERO_PROF_GATHER_LN,
               launch_gather_ln_modulate(d_x, ga, d_idx, shift2, scale2, mod_ld, c->ws_a, B, N, n_sel, D, 1e-5f,
@@ -392,6 +403,7 @@ void hero_destroy(hero_ctx* c) {
   if (c->stream) cudaStreamSynchronize(c->stream); else cudaDeviceSynchronize();
   if (c->copy_stream) { cudaStreamSynchronize(c->copy_stream); cudaStreamDestroy(c->copy_stream); }
   for (cudaEvent_t e : c->piece_done) if (e) cudaEventDestroy(e);
+  if (c->x_uploaded) cudaEventDestroy(c->x_uploaded);
   for (void* p : c->allocs) cudaFree(p);
   for (auto& sp : c->spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
   for (auto& sp : c->span_pool) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
@@ -697,17 +709,40 @@ static int step_impl(hero_ctx* c, int step, void* d_x, const void* d_temb, void*
 int hero_step_host(hero_ctx* c, int step, void* h_x, const void* h_temb) {
   if (!c || !h_x || !h_temb) return HERO_ERR_ARG;
   const size_t xb = (size_t)c->elems * c->esz, tb = (size_t)c->cfg.batch * c->cfg.temb_dim * c->esz;
-  HERO_CUDA_TRY(cudaMemcpyAsync(c->x_stage, h_x, xb, cudaMemcpyHostToDevice, c->stream));
-  HERO_CUDA_TRY(cudaMemcpyAsync(c->temb_stage, h_temb, tb, cudaMemcpyHostToDevice, c->stream));
   if (!c->copy_stream) {
     HERO_CUDA_TRY(cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
     for (cudaEvent_t& e : c->piece_done) HERO_CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+    HERO_CUDA_TRY(cudaEventCreateWithFlags(&c->x_uploaded, cudaEventDisableTiming));
+  }
+  // A cached step whose first block refreshes something, with x in pinned (device-visible) host memory: the
+  // upload of x goes to the copy stream and the first block's LayerNorm reads its rows from the host copy, so
+  // that its GEMMs and attention run while the rest of x is still on its way.
+  const void* h_alias = nullptr;
+  const hero_config& g = c->cfg;
+  if (step >= 0 && !is_full(g, step) && g.n_shallow > 0 && c->n_full > 0 &&
+      n_sel_for_call(c, c->blk[0].calls) > 0) {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, h_x) == cudaSuccess && at.type == cudaMemoryTypeHost && at.devicePointer)
+      h_alias = at.devicePointer;
+    else
+      cudaGetLastError();                    // pageable memory: not an error, just no shortcut
+  }
+  HERO_CUDA_TRY(cudaMemcpyAsync(c->temb_stage, h_temb, tb, cudaMemcpyHostToDevice, c->stream));
+  if (h_alias) {
+    HERO_CUDA_TRY(cudaMemcpyAsync(c->x_stage, h_x, xb, cudaMemcpyHostToDevice, c->copy_stream));
+    HERO_CUDA_TRY(cudaEventRecord(c->x_uploaded, c->copy_stream));
+    c->first_rows_src = h_alias;
+    c->wait_x_upload = true;
+  } else {
+    HERO_CUDA_TRY(cudaMemcpyAsync(c->x_stage, h_x, xb, cudaMemcpyHostToDevice, c->stream));
   }
   bool copied = false;
   const int rc = step_impl(c, step, c->x_stage, c->temb_stage, h_x, &copied);
-  if (rc != HERO_OK) {                       // leave no copy in flight behind an error
+  c->first_rows_src = nullptr;
+  if (rc != HERO_OK || c->wait_x_upload) {   // leave no copy in flight behind an error (or an unused upload)
+    c->wait_x_upload = false;
     cudaStreamSynchronize(c->copy_stream);
-    return rc;
+    if (rc != HERO_OK) return rc;
   }
   if (!copied) HERO_CUDA_TRY(cudaMemcpyAsync(h_x, c->x_stage, xb, cudaMemcpyDeviceToHost, c->stream));
   HERO_CUDA_TRY(cudaStreamSynchronize(c->stream));

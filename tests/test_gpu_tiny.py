@@ -50,18 +50,23 @@ def test_tiny_ten_steps_match_oracle():
     print("worst rel-L2 over 10 steps:", worst)
 
 
-def test_tiny_host_entry_point_matches_device_entry_point():
+@pytest.mark.parametrize("pinned", [True, False])
+def test_tiny_host_entry_point_matches_device_entry_point(pinned):
+    """Pinned host buffers take the overlapped route (first block's rows read from the host copy while x uploads,
+    finished pieces copied back behind the deep pass); pageable ones the plain copy-in, step, copy-out."""
     cfgd = S.CONFIGS["tiny"]
     _, hero_a, w = make_pair(cfgd)
     _, hero_b, _ = make_pair(cfgd, w)
     x0 = torch.from_numpy(S.tokens(cfgd))
-    for s in range(4):
+    for s in range(5):
         temb = torch.from_numpy(S.temb(cfgd, s))
         xd = x0.cuda()
         hero_a.hero_step(s, xd, temb.cuda())
-        xh = x0.clone().pin_memory()
-        hero_b.hero_step_host(s, xh, temb.pin_memory())
-        assert torch.equal(xd.cpu(), xh)
+        xh = x0.clone().pin_memory() if pinned else x0.clone()
+        assert xh.is_pinned() == pinned
+        hero_b.hero_step_host(s, xh, temb.pin_memory() if pinned else temb.clone())
+        assert torch.equal(xd.cpu(), xh), s
+    hero_a.hero_check_status(); hero_b.hero_check_status()
     hero_a.close(); hero_b.close()
 
 
