@@ -37,6 +37,8 @@ from workloads import synthetic as S  # noqa: E402
 METRIC = "hero_cached_step_tokens_per_s"
 ATTENTION_TRAFFIC_RATIO = 1.002   # dram__bytes_read+write / algorithmic bytes of tc_attention_kernel (ncu, small case)
 UNIT = "tokens/s"
+NOMINAL_BF16_TFLOPS = 2250.0      # dense bf16, the figure the 60 % target is stated against
+NOMINAL_HBM_GBS = 8000.0          # the figure the 70 % target is stated against
 
 
 # --------------------------------------------------------------------------- helpers
@@ -63,9 +65,12 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._pump, daemon=True)
             self.thread.start()
+            t0 = time.time()
+            while not self.lines and time.time() - t0 < 2.0:      # the first sample marks the loop as running
+                time.sleep(0.01)
         except OSError:
             self.proc = None
 
@@ -159,6 +164,11 @@ class OracleSample:
         return total, detail
 
 
+ORACLE_SAMPLE_ROWS = 128      # rows whose branch outputs the oracle computes per sampled step (both arms)
+ORACLE_SAMPLE_TEXT = ("one shallow block refreshed on its real selection (K/V of every selected row, branch outputs of "
+                      "%d rows, scaled to all) + one deep block extrapolated, scaled by block counts" % ORACLE_SAMPLE_ROWS)
+
+
 def cpu_cores_used():
     try:
         from threadpoolctl import threadpool_info
@@ -183,12 +193,11 @@ def run_reference(args, cfg, rank, world):
     vals = []
     sample_obj = OracleSample(cfg)
     for i in range(args.warmup + args.steps):
-        sec, detail = sample_obj.step_seconds(sample_rows=128)
+        sec, detail = sample_obj.step_seconds(sample_rows=ORACLE_SAMPLE_ROWS)
         if i >= args.warmup:
             vals.append(sec)
     sec = statistics.mean(vals)
-    sample = ("per step: one shallow block refreshed on its real selection (K/V of every selected row, branch "
-              "outputs of 128 rows, scaled to all) + one deep block extrapolated, scaled by block counts")
+    sample = "per step: " + ORACLE_SAMPLE_TEXT
     line = {"impl": "reference", "metric": METRIC, "value": tokens / sec, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
@@ -334,14 +343,22 @@ def run_hero(args, cfg, rank, world, local_rank):
         # algorithmic bytes (K and V once, Q in, O out); the traffic grows in proportion with those, so the
         # full launch is that ratio times its own algorithmic bytes
         alg_bytes = 2 * B * N * D * 2 + 2 * B * n_sel * D * 2
+        gemm_tf = fl["gemm"] / (gemm_ms_blk * 1e-3) / 1e12
         roofline = {"kernel": "tc_attention_kernel", "bound": "tensor", "achieved": achieved, "peak": peak,
-                    "unit": "TFLOP/s", "frac": achieved / peak, "traffic": ATTENTION_TRAFFIC_RATIO * alg_bytes,
+                    "unit": "TFLOP/s", "frac": achieved / peak, "frac_of_burst": achieved / peaks["bf16_tflops"],
+                    "frac_of_2250": achieved / NOMINAL_BF16_TFLOPS, "traffic": ATTENTION_TRAFFIC_RATIO * alg_bytes,
                     "traffic_source": "ncu small case (profiles/tc_attention_small_q768.md) scaled by algorithmic bytes",
                     "peak_source": peaks["source"] + " (sustained cuBLAS bf16)",
                     "flops_per_launch": fl["attention"], "ms_per_launch": att_ms,
-                    "gemm": {"achieved": fl["gemm"] / (gemm_ms_blk * 1e-3) / 1e12, "unit": "TFLOP/s",
-                             "frac": fl["gemm"] / (gemm_ms_blk * 1e-3) / 1e12 / peak,
-                             "flops_per_block": fl["gemm"], "ms_per_block": gemm_ms_blk}}
+                    "gemm": {"achieved": gemm_tf, "unit": "TFLOP/s", "frac": gemm_tf / peak,
+                             "frac_of_burst": gemm_tf / peaks["bf16_tflops"], "frac_of_2250": gemm_tf / NOMINAL_BF16_TFLOPS,
+                             "flops_per_block": fl["gemm"], "ms_per_block": gemm_ms_blk},
+                    "refresh_block": {"achieved": (fl["gemm"] + fl["attention"]) / ((gemm_ms_blk + att_ms) * 1e-3) / 1e12,
+                                      "unit": "TFLOP/s",
+                                      "frac": (fl["gemm"] + fl["attention"]) / ((gemm_ms_blk + att_ms) * 1e-3) / 1e12 / peak,
+                                      "frac_of_2250": (fl["gemm"] + fl["attention"]) / ((gemm_ms_blk + att_ms) * 1e-3) / 1e12
+                                                      / NOMINAL_BF16_TFLOPS,
+                                      "note": "the four GEMMs and the attention of one refresh block together"}}
         if breakdown["extrapolate"]["launches_per_step"]:
             # all deep blocks in one pass per launch: four history tensors read per block, x read and written
             # once per launch
@@ -350,6 +367,7 @@ def run_hero(args, cfg, rank, world, local_rank):
             ext_bytes = B * N * D * 2 * (4 * n_deep + 2 * breakdown["extrapolate"]["launches_per_step"])
             gbs = ext_bytes / (ext_ms * 1e-3) / 1e9
             roofline["extrapolate"] = {"achieved": gbs, "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                                       "frac_of_8tbs": gbs / NOMINAL_HBM_GBS,
                                        "ms_per_step": ext_ms, "bytes_per_step": ext_bytes, "blocks": n_deep}
 
     # end to end through the host entry point: pinned host buffers, H2D + step + D2H per call
@@ -358,15 +376,21 @@ def run_hero(args, cfg, rank, world, local_rank):
     n_e2e = max(2, min(args.steps, 5))
     hero.hero_step_host(step, h_x, h_t); step += 1
     torch.cuda.synchronize()
+    first_rows = []                      # rows the first refresh block reads straight from the pinned buffer
     t0 = time.perf_counter()
     for _ in range(n_e2e):
+        first_rows.append(hero.hero_next_n_sel(0) if cfg["n_shallow"] else 0)
         hero.hero_step_host(step, h_x, h_t); step += 1
     e2e_s = (time.perf_counter() - t0) / n_e2e
     e2e_s = max_over_ranks(e2e_s, dist, device)
     xb = h_x.numel() * h_x.element_size()
     tb = h_t.numel() * h_t.element_size()
+    zero_copy = int(statistics.mean(first_rows) * B * D * h_x.element_size())
     e2e = {"value": whole_job_throughput(tokens, world, e2e_s * 1e3), "unit": UNIT, "ms_per_step": e2e_s * 1e3,
-           "h2d_bytes_per_step": xb + tb, "d2h_bytes_per_step": xb}
+           "h2d_bytes_per_step": xb + tb + zero_copy, "d2h_bytes_per_step": xb,
+           "h2d_copy_bytes_per_step": xb + tb, "h2d_zero_copy_bytes_per_step": zero_copy,
+           "note": "h2d = the upload of x and temb plus the rows of x that the first refresh block's LayerNorm reads "
+                   "directly from the pinned host buffer over PCIe while the upload is under way"}
     hero.hero_check_status()
     mem = hero.hero_device_bytes()
     hero.close()
@@ -411,16 +435,27 @@ def run_hero(args, cfg, rank, world, local_rank):
             base_qk["note"] = ("qk_norm=1, rope=1: the base model's per-head LayerNorm and 3-D rotary embedding of the "
                                "fresh q and k rows (one extra HBM-bound pass per refresh block)")
 
+    kernels_record = None
+    if rank == 0 and world == 1 and not args.no_kernels:
+        recs, k_clocks = config2_kernels(H, device, measured_peaks(), iters=20, warm=3)
+        kernels_record = {"workload": "isolated kernels on [2, 17776, 3072] bf16, index lists at 10/25/50 % of a 13x30x45 "
+                                      "grid (2x2 patches)",
+                          "timing": "each kernel alone, CUDA events, median of 20 calls, L2 flushed before every call",
+                          "clocks": k_clocks, "kernels": recs}
+
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         del weights
         torch.cuda.empty_cache()
-        sec, detail = OracleSample(cfg).step_seconds(sample_rows=256)
+        # the same sample and estimator as `--impl reference`: one untimed pass (BLAS threads, page faults), then
+        # the mean of two
+        smp = OracleSample(cfg)
+        smp.step_seconds(sample_rows=ORACLE_SAMPLE_ROWS)
+        runs = [smp.step_seconds(sample_rows=ORACLE_SAMPLE_ROWS) for _ in range(2)]
+        sec = statistics.mean(r[0] for r in runs)
         cpu_baseline = {"value": tokens / sec, "unit": UNIT, "cores": cpu_cores_used(), "kind": "oracle",
-                        "sample": "one shallow block refreshed on its real selection (K/V of all selected rows, "
-                                  "branch outputs of 256 rows scaled to all) + one deep block extrapolated, scaled "
-                                  f"to {cfg['n_shallow']} + {cfg['n_blocks'] - cfg['n_shallow']} blocks; "
-                                  f"{detail['cpu_work_s']:.1f} s of CPU work",
+                        "sample": ORACLE_SAMPLE_TEXT + "; mean of 2 samples after 1 untimed, "
+                                  f"{sum(r[1]['cpu_work_s'] for r in runs):.1f} s of timed CPU work",
                         "ms_per_step": sec * 1e3}
 
     if rank == 0:
@@ -457,6 +492,8 @@ def run_hero(args, cfg, rank, world, local_rank):
                                         "frac": ach_exp / peak_exp,
                                         "note": "secondary bound of the attention kernel at head_dim 64"}
             line["roofline"] = roofline
+        if kernels_record:
+            line["kernels"] = kernels_record
         if cpu_baseline:
             line["cpu_baseline"] = cpu_baseline
         print(json.dumps(line))
@@ -481,6 +518,73 @@ def _time_flushed(fn, iters, warmup, flush):
             ts.append(e0.elapsed_time(e1))
     return statistics.median(ts)
 
+
+
+def config2_kernels(H, dev, peaks, iters=20, warm=3, want=None):
+    """The isolated-kernel workload (feature cache [2, 17776, 3072] bf16, index lists at 10 / 25 / 50 % drawn by
+    the library's own sampler on the 13x30x45 grid with 2x2 patches): Eq. 5 alone, row gather and scatter, and
+    the gather + LayerNorm + modulate prologue, each timed alone with CUDA events, L2 flushed before every call,
+    median of `iters` calls, clocks sampled over the whole group.  Returns (records, clocks)."""
+    want = want or (lambda name: True)
+    cfg = dict(S.CONFIGS["kernels"])
+    B, N, D = cfg["batch"], S.n_rows(cfg), cfg["hidden"]
+    bf = torch.bfloat16
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    out = {}
+
+    def rnd(*shape, std=1.0):
+        return (torch.randn(*shape, device=dev) * std).to(bf)
+
+    def hbm(name, ms, nbytes, **extra):
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        out[name] = dict(ms=ms, bytes=nbytes, achieved=gbs, unit="GB/s", frac=gbs / peaks["hbm_gbs"],
+                         frac_of_8tbs=gbs / NOMINAL_HBM_GBS, bound="hbm", **extra)
+
+    # index lists from the library's own sampler (a context with a one-head block: only geometry matters)
+    lists = {}
+    small_cfg = dict(cfg, hidden=64, n_heads=1, ffn_dim=64, temb_dim=64, n_blocks=1, n_shallow=1)
+    w = [{k: torch.zeros(s_, device=dev, dtype=bf) for k, s_ in S.weight_shapes(small_cfg).items()}]
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    for num, den in ((1, 10), (1, 4), (1, 2)):
+        hero = H.Hero(dict(small_cfg, ratio_num=num, ratio_den=den), w)
+        idx = torch.empty(S.n_video(cfg), dtype=torch.int32, device=dev)
+        n = hero.hero_select_tokens(0, idx)
+        lists[f"{num}/{den}"] = idx[:n].clone()
+        if want("select") and (num, den) == (1, 4):
+            ms = _time_flushed(lambda: hero.hero_select_tokens(0, idx), iters, warm, flush)
+            out["select_25"] = dict(ms=ms, tokens=S.n_video(cfg), bound="latency",
+                                    note="integer work on 35 KB of counters; no bandwidth figure applies")
+        hero.close()
+    if want("extrapolate"):
+        a, b_, o = rnd(B, N, D), rnd(B, N, D), torch.empty(B, N, D, device=dev, dtype=bf)
+        hbm("extrapolate", _time_flushed(lambda: H.hero_extrapolate(a, b_, o, 4, 5), iters, warm, flush), 3 * a.numel() * 2)
+        del a, b_, o
+    if want("gather") or want("scatter") or want("gather_ln"):
+        src = rnd(B, N, D)
+        add = rnd(B, N, D, std=0.3)
+        mod = torch.randn(B, 4 * D, device=dev) * 0.5
+        for key, idx in lists.items():
+            comp = torch.empty(B, idx.numel(), D, device=dev, dtype=bf)
+            nbytes = 2 * B * idx.numel() * D * 2 + 4 * idx.numel()
+            if want("gather"):
+                hbm(f"gather_{key}", _time_flushed(lambda: H.hero_gather_rows(src, idx, comp), iters, warm, flush),
+                    nbytes, rows=idx.numel())
+            if want("scatter"):
+                hbm(f"scatter_{key}", _time_flushed(lambda: H.hero_scatter_rows(comp, idx, src), iters, warm, flush),
+                    nbytes, rows=idx.numel())
+            if want("gather_ln"):
+                # the prologue of the attention branch (rows in, rows out) and of the FFN branch (two rows in)
+                hbm(f"gather_ln_{key}", _time_flushed(
+                    lambda: H.hero_gather_ln_modulate(src, None, idx, mod[:, :D], mod[:, D:2 * D], comp), iters, warm, flush),
+                    nbytes, rows=idx.numel())
+                hbm(f"gather_ln_add_{key}", _time_flushed(
+                    lambda: H.hero_gather_ln_modulate(src, add, idx, mod[:, :D], mod[:, D:2 * D], comp), iters, warm, flush),
+                    nbytes + B * idx.numel() * D * 2, rows=idx.numel())
+        del src, add
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    return out, clocks
 
 def run_kernels(args):
     """Each kernel of the cached step alone, at the shapes of the isolated-kernel and one-block
@@ -517,27 +621,10 @@ def run_kernels(args):
                          frac_of_sustained=tf / peaks["bf16_tflops_sustained"], frac_of_2250=tf / 2250.0,
                          bound="tensor", **extra)
 
-    # index lists from the library's own sampler (a context with a one-head block: only geometry matters)
-    lists = {}
-    if want("gather") or want("scatter") or want("select"):
-        small_cfg = dict(cfg, hidden=64, n_heads=1, ffn_dim=64, temb_dim=64, n_blocks=1, n_shallow=1)
-        w = [{k: torch.zeros(s, device=dev, dtype=bf) for k, s in S.weight_shapes(small_cfg).items()}]
-        for num, den in ((1, 10), (1, 4), (1, 2)):
-            hero = H.Hero(dict(small_cfg, ratio_num=num, ratio_den=den), w)
-            idx = torch.empty(S.n_video(cfg), dtype=torch.int32, device=dev)
-            n = hero.hero_select_tokens(0, idx)
-            lists[f"{num}/{den}"] = idx[:n].clone()
-            if want("select") and (num, den) == (1, 4):
-                ms = _time_flushed(lambda: hero.hero_select_tokens(0, idx), iters, warm, flush)
-                out["select_25"] = dict(ms=ms, tokens=S.n_video(cfg), bound="latency",
-                                        note="integer work on 35 KB of counters; no bandwidth figure applies")
-            hero.close()
-
-    if want("extrapolate"):
-        a, b_, o = rnd(B, N, D), rnd(B, N, D), torch.empty(B, N, D, device=dev, dtype=bf)
-        ms = _time_flushed(lambda: H.hero_extrapolate(a, b_, o, 4, 5), iters, warm, flush)
-        hbm("extrapolate", ms, 3 * a.numel() * 2)
-        del a, b_, o
+    sampler = ClockSampler(torch.cuda.current_device())
+    c2, c2_clocks = config2_kernels(H, dev, peaks, iters, warm, want)
+    out.update(c2)
+    sampler.start()
     if want("diagnostics"):
         a, b_, c_ = rnd(B, N, D), rnd(B, N, D), rnd(B, N, D)
         mom = torch.zeros(2, dtype=torch.float64, device=dev)
@@ -546,18 +633,6 @@ def run_kernels(args):
         ms = _time_flushed(lambda: H.hero_extrapolation_error(a, b_, c_, 2, 5, mom), iters, warm, flush)
         hbm("extrapolation_error", ms, 3 * a.numel() * 2)
         del a, b_, c_
-    if want("gather") or want("scatter"):
-        src = rnd(B, N, D)
-        for key, idx in lists.items():
-            comp = torch.empty(B, idx.numel(), D, device=dev, dtype=bf)
-            nbytes = 2 * B * idx.numel() * D * 2 + 4 * idx.numel()
-            if want("gather"):
-                hbm(f"gather_{key}", _time_flushed(lambda: H.hero_gather_rows(src, idx, comp), iters, warm, flush),
-                    nbytes, rows=idx.numel())
-            if want("scatter"):
-                hbm(f"scatter_{key}", _time_flushed(lambda: H.hero_scatter_rows(comp, idx, src), iters, warm, flush),
-                    nbytes, rows=idx.numel())
-        del src
     if want("attention"):
         cases = [(1, 768)] if args.small else [(B, 1755), (B, 4387), (B, 8775)]
         for bb, nq in cases:
@@ -638,9 +713,12 @@ def run_kernels(args):
             fl = refresh_flops(bcfg, state["n"])
             tensor(f"refresh_block_{num}/{den}", ms, fl["gemm"] + fl["attention"], n_sel=state["n"])
             hero.close()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
     print(json.dumps({"workload": "kernels", "small": bool(args.small), "iters": iters, "timing":
                       "CUDA events, median, L2 flushed by a 256 MiB write + read before every call",
-                      "peaks": peaks, "kernels": out}))
+                      "peaks": peaks, "clocks": {"isolated_hbm_kernels": c2_clocks, "tensor_and_block_kernels": clocks},
+                      "kernels": out}))
 
 
 def main():
@@ -651,10 +729,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="hero", choices=["hero", "reference"])
     ap.add_argument("--workload", default="dit42", choices=["dit42", "aether", "paper_hp", "tiny", "kernels"])
-    ap.add_argument("--only", default="", help="kernels workload: comma list of select,extrapolate,gather,scatter,"
+    ap.add_argument("--only", default="", help="kernels workload: comma list of select,extrapolate,gather,scatter,gather_ln,"
                                                "attention,gemm,deep,deep_group,block,diagnostics")
     ap.add_argument("--small", action="store_true", help="kernels workload: profiler-sized tensor-core cases")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-kernels", action="store_true", help="skip the isolated-kernel record of the default line")
     ap.add_argument("--cfg-split", action="store_true",
                     help="with --gpus N: split the batch items of ONE problem over the ranks instead of running N problems")
     ap.add_argument("--no-collapse", action="store_true", help="skip the variant runs (collapsed deep stack, refreshed-rows-only attention)")

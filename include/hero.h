@@ -18,8 +18,11 @@
  *     (frame, y, x) order.  Run dtype (fp32 or bf16) applies to x, temb, weights
  *     and caches alike.
  *   - Weight matrices are row-major [out_features, in_features] (K contiguous).
- *     Device pointers must be 16-byte aligned; in bf16 mode hidden, ffn_dim and
- *     temb_dim must be multiples of 8 and head_dim must be 64.
+ *     Device pointers must be 16-byte aligned; in bf16 mode hidden and ffn_dim must be
+ *     multiples of 32, temb_dim a multiple of 8 and head_dim must be 64.  batch * temb_dim
+ *     is at most 12288, and hidden at most 12288 unless the run is bf16 with hidden 1024,
+ *     2048, 3072 or 4096 (shared-memory limits of the streaming kernels); hero_init
+ *     refuses anything else with HERO_ERR_ARG / HERO_ERR_ALIGN.
  *   - All work is enqueued on the CUDA stream given to hero_init; no call
  *     synchronises the device unless stated.  Calls on one context must not
  *     overlap in time.  hero_step, hero_refresh_block and the extrapolation calls
@@ -97,12 +100,15 @@ typedef struct hero_block_weights {
 
 /* ---- context ------------------------------------------------------------- */
 
-/* Validate cfg, allocate caches (K, V, G_attn, G_ffn per shallow block; two history
- * slots x two branches per deep block), age counters, workspace and TMA descriptors
+/* Algorithm 1's state: validate cfg (the hyper-parameters of Sec. 5.1: K = n_shallow, M = full_interval,
+ * R, p_h x p_w), allocate the caches Algorithm 1 writes in its "initial caching" part (K, V, G_attn, G_ffn
+ * per shallow block; two history slots x two branches per deep block, which carry the same information as
+ * the G and Delta G of Sec. 4.4), the age counters of Sec. 4.3's tracking, workspace and TMA descriptors
  * on the current device.  blocks[n_blocks] is copied; the weights it points to are
  * not.  cuda_stream is a cudaStream_t (NULL = legacy default stream). */
 int hero_init(hero_ctx **out, const hero_config *cfg, const hero_block_weights *blocks, void *cuda_stream);
-/* Forget all cached state (ages, call counters, step history); memory is kept. */
+/* Back to the state before Algorithm 1's first step: forget all cached state (ages, call counters, step
+ * history, which caches hold a full pass); memory is kept. */
 int hero_reset(hero_ctx *ctx);
 void hero_destroy(hero_ctx *ctx);
 const char *hero_strerror(int code);
@@ -149,7 +155,9 @@ int hero_next_n_sel(const hero_ctx *ctx, int block);
  * FFN (GELU-tanh) rows into G_ffn -> x += G_ffn.  d_idx == NULL with n_sel == N is the full
  * pass ("initial caching"): all rows, ages reset, deep blocks rotate their history slots.
  * n_sel == 0 refreshes nothing and only adds the cached branches (d_idx is not read).
- * d_x [batch,N,hidden] is updated in place; d_temb is [batch, temb_dim]. */
+ * d_x [batch,N,hidden] is updated in place; d_temb is [batch, temb_dim].
+ * A partial or empty refresh merges with what the block's caches hold, so the block must have had a full
+ * pass first (or all four caches planted with hero_state_set): HERO_ERR_STATE otherwise. */
 int hero_refresh_block(hero_ctx *ctx, int block, void *d_x, const void *d_temb,
                        const int *d_idx, int n_sel);
 
@@ -205,29 +213,50 @@ int hero_extrapolation_error(const void *d_g_prev, const void *d_g_last, const v
 /* Eq. 5 alone: out = g_last + (g_last - g_prev) * k/d over n_elem elements. */
 int hero_extrapolate(const void *d_g_prev, const void *d_g_last, void *d_out, long long n_elem,
                      int k, int d, int dtype, void *stream);
-/* dst[b, i, :] = src[b, idx[i], :] for b < B, i < n_sel; src is [B,N,D], dst [B,n_sel,D]. */
+/* The gather of the selected rows S(z) that Eq. 3's F(S(z), ...) starts from:
+ * dst[b, i, :] = src[b, idx[i], :] for b < B, i < n_sel; src is [B,N,D], dst [B,n_sel,D]. */
 int hero_gather_rows(const void *d_src, const int *d_idx, void *d_dst, int B, int N, int n_sel,
                      int D, int dtype, void *stream);
 /* dst[b, idx[i], :] = src[b, i, :]; other rows of dst are not touched (Eq. 3's merge). */
 int hero_scatter_rows(const void *d_src, const int *d_idx, void *d_dst, int B, int N, int n_sel,
                       int D, int dtype, void *stream);
+/* The prologue of Eq. 2 alone (LayerNorm of Sec. 3's block with the adaLN scale and shift the paper's
+ * equations leave out "for clarity"), fused with the gather of the selected rows:
+ * out[b, i, :] = LN(x[b, idx[i], :] + add[b, idx[i], :]) * (1 + scale[b, :]) + shift[b, :], LN = zero mean,
+ * unit (biased) variance over the D features, eps 1e-5, statistics in fp32.  d_x and d_add (may be NULL)
+ * are [B,N,D] in `dtype`; d_idx int32[n_sel] (NULL = rows 0..n_sel-1); d_shift, d_scale fp32 with
+ * batch stride mod_ld (>= D; float4 loads are used when mod_ld % 4 == 0 and both are 16-byte aligned);
+ * d_out [B,n_sel,D] compact, in `dtype`.  HERO_ERR_ARG / HERO_ERR_ALIGN before anything is launched. */
+int hero_gather_ln_modulate(const void *d_x, const void *d_add, const int *d_idx, const float *d_shift,
+                            const float *d_scale, int mod_ld, void *d_out, int B, int N, int n_sel, int D,
+                            int dtype, void *stream);
 /* C[M,N] = A[M,K] * W[N,K]^T + bias[N] in bf16 with fp32 accumulation on the tensor cores
  * (act = 1 applies GELU-tanh).  The GEMM of the refresh path, exposed for tests and timing. */
 int hero_gemm_bf16(const void *d_a, const void *d_w, const void *d_bias, void *d_c,
                    int M, int N, int K, int act, void *stream);
 /* O[b,i,h,:] = softmax_j(Q[b,i,h,:] . K[b,j,h,:] / sqrt(head_dim)) V[b,j,h,:], j over all N
- * rows; Q,O are [B,n_q,heads*64] bf16, K,V are [B,N,heads*64] bf16.  No score matrix is stored. */
+ * rows; Q,O are [B,n_q,heads*64] bf16, K,V are [B,N,heads*64] bf16.  No score matrix is stored
+ * (Sec. 4.3: the refresh stays compatible with FlashAttention-style kernels).  Two launches: a fast
+ * kernel that scales every row by the maximum of its first 96 scores for good, and a second one that
+ * recomputes, with a running maximum, the thread blocks in which some later score exceeded that maximum
+ * by more than 2^100 (no such block on ordinary inputs: it then returns at once). */
 int hero_attention_bf16(const void *d_q, const void *d_k, const void *d_v, void *d_o,
                         int B, int n_q, int N, int heads, void *stream);
+/* The same result from the second kernel alone (running maximum, accumulator rescaled in place when a
+ * tile exceeds it by 2^8): what hero_attention_bf16 falls back to, exposed for tests and for inputs
+ * known to have an extreme dynamic range. */
+int hero_attention_bf16_safe(const void *d_q, const void *d_k, const void *d_v, void *d_o,
+                             int B, int n_q, int N, int heads, void *stream);
 
 /* hero_attention_bf16 without any allocation (the paper has no counterpart: this entry point
  * exists for the sake of callers, not of the method).  hero_attention_bf16 obtains its status
  * word with cudaMalloc on first use; a caller that must never enter the CUDA allocator - a
  * serving loop that cannot take the device-wide synchronisation cudaMalloc/cudaFree imply, a
  * process whose framework already owns all device memory, code running where allocation is
- * forbidden - calls this instead.  Same arguments and same result (bit for bit); its scratch is
- * a fixed 64.25 KiB array inside the library image, present on every GPU that loads the library
- * until the process exits.
+ * forbidden - calls this instead.  Same arguments and same result (bit for bit); its scratch (the
+ * give-up counter and the per-thread-block words through which the fast kernel hands blocks to the
+ * fallback kernel) is a fixed 64.25 KiB array inside the library image, present on every GPU that
+ * loads the library until the process exits.
  *   - Limit: ceil(n_q / 256) * heads * B <= 16384 (one scratch word per thread block); beyond
  *     that nothing is launched, HERO_ERR_CAP is returned and hero_last_cuda_error() says why.
  *   - The first call on each device resolves the array's device address and sets the kernel's
@@ -240,10 +269,26 @@ int hero_attention_bf16(const void *d_q, const void *d_k, const void *d_v, void 
  * Calls cudaMalloc, cudaFree or any allocating library routine: never. */
 int hero_attention_bf16_static(const void *d_q, const void *d_k, const void *d_v, void *d_o,
                                int B, int n_q, int N, int heads, void *stream, int *h_gave_up);
+/* The verdict of the latest hero_attention_bf16_static call on the current device, for a caller that
+ * passed h_gave_up = NULL to keep that call asynchronous and still must not allocate (hero_isolated_status
+ * watches a different word, one that comes from cudaMalloc).  Waits for everything queued on `stream`,
+ * then stores in *h_gave_up (host, required) the number of thread blocks of that call which gave up on a
+ * bounded wait and, when h_records is given, one word per thread block i < n_records (0 = finished, 2 = gave
+ * up; n_records <= 16384).  Returns HERO_ERR_TIMEOUT if the count is not 0.  The paper has no counterpart. */
+int hero_attention_bf16_static_status(void *stream, int *h_gave_up, int *h_records, int n_records);
 
 /* Synchronise `stream` and return HERO_ERR_TIMEOUT if hero_gemm_bf16 / hero_attention_bf16 gave
- * up on a bounded device-side wait since the last poll, else HERO_OK. */
+ * up on a bounded device-side wait since the last poll, else HERO_OK.  The word that is polled lives
+ * on the device that is current at the call (one per device). */
 int hero_isolated_status(void *stream);
+/* Self-test of the give-up path (no counterpart in the paper).  Every device-side wait of the tensor-core
+ * kernels is bounded: when its budget runs out the kernel raises a status word and returns instead of
+ * spinning.  This call runs exactly that on purpose, harmlessly: ONE thread block, no TMA, no tensor
+ * memory, waits budget_us microseconds (1..100000) through the same helper on a barrier that nobody
+ * completes, raises the word and returns.  With ctx given the word and the stream are the context's
+ * (the next hero_check_status returns HERO_ERR_TIMEOUT once, then HERO_OK again); with ctx = NULL they
+ * are the isolated calls' word and `stream` (hero_isolated_status reports it the same way). */
+int hero_selftest_wait_timeout(hero_ctx *ctx, int budget_us, void *stream);
 
 /* ---- state access for tests and checkpoints -------------------------------- */
 #define HERO_STATE_AGES     0   /* u16[n_video] */

@@ -25,7 +25,8 @@ EXPORTS = [
     "hero_init", "hero_reset", "hero_destroy", "hero_strerror", "hero_check_status", "hero_last_cuda_error",
     "hero_device_bytes", "hero_launch_count", "hero_profile_begin", "hero_profile_end", "hero_select_tokens", "hero_next_n_sel", "hero_refresh_block",
     "hero_extrapolate_block", "hero_extrapolate_deep_stack", "hero_step", "hero_step_host", "hero_is_full_step", "hero_extrapolate",
-    "hero_gather_rows", "hero_scatter_rows", "hero_gemm_bf16", "hero_attention_bf16", "hero_attention_bf16_static", "hero_isolated_status",
+    "hero_gather_rows", "hero_scatter_rows", "hero_gemm_bf16", "hero_attention_bf16", "hero_attention_bf16_safe", "hero_attention_bf16_static", "hero_attention_bf16_static_status",
+    "hero_isolated_status", "hero_selftest_wait_timeout", "hero_gather_ln_modulate",
     "hero_state_get", "hero_state_set", "hero_second_difference_moments", "hero_extrapolation_error",
 ]
 
@@ -91,8 +92,12 @@ def load() -> C.CDLL:
         "hero_scatter_rows": (i, [vp, vp, vp, i, i, i, i, i, vp]),
         "hero_gemm_bf16": (i, [vp, vp, vp, vp, i, i, i, i, vp]),
         "hero_attention_bf16": (i, [vp, vp, vp, vp, i, i, i, i, vp]),
+        "hero_attention_bf16_safe": (i, [vp, vp, vp, vp, i, i, i, i, vp]),
         "hero_attention_bf16_static": (i, [vp, vp, vp, vp, i, i, i, i, vp, ip]),
+        "hero_attention_bf16_static_status": (i, [vp, ip, ip, i]),
         "hero_isolated_status": (i, [vp]),
+        "hero_selftest_wait_timeout": (i, [vp, i, vp]),
+        "hero_gather_ln_modulate": (i, [vp, vp, vp, vp, vp, i, vp, i, i, i, i, i, vp]),
         "hero_second_difference_moments": (i, [vp, vp, vp, ll, i, vp, vp]),
         "hero_extrapolation_error": (i, [vp, vp, vp, ll, i, i, i, vp, vp]),
         "hero_state_get": (i, [vp, i, i, vp, ll]),
@@ -218,6 +223,10 @@ class Hero:
     def hero_check_status(self):
         _check(self.lib.hero_check_status(self.ctx), "hero_check_status")
 
+    def hero_selftest_wait_timeout(self, budget_us: int = 50):
+        """Make one bounded device-side wait run out on purpose (it raises this context's status word)."""
+        _check(self.lib.hero_selftest_wait_timeout(self.ctx, budget_us, None), "hero_selftest_wait_timeout")
+
     def hero_device_bytes(self) -> int:
         return self.lib.hero_device_bytes(self.ctx)
 
@@ -320,6 +329,16 @@ def hero_attention_bf16(q, k, v, o, heads: int):
     return o
 
 
+def hero_attention_bf16_safe(q, k, v, o, heads: int):
+    """The fallback attention kernel alone (running maximum with in-place rescaling)."""
+    _require_cuda()
+    B, n_q, _ = q.shape
+    N = k.shape[1]
+    _check(load().hero_attention_bf16_safe(_ptr(q), _ptr(k), _ptr(v), _ptr(o), B, n_q, N, heads, _stream()),
+           "hero_attention_bf16_safe")
+    return o
+
+
 def hero_attention_bf16_static(q, k, v, o, heads: int, check: bool = True):
     """hero_attention_bf16 for callers that must not allocate device memory: the kernel's scratch is a
     fixed array inside the library.  With check=True the call waits for the result and raises if any
@@ -333,8 +352,36 @@ def hero_attention_bf16_static(q, k, v, o, heads: int, check: bool = True):
     return o
 
 
+def hero_attention_bf16_static_status(n_records: int = 0):
+    """(thread blocks that gave up, their per-block records) of the latest hero_attention_bf16_static call."""
+    _require_cuda()
+    gave_up = C.c_int(-1)
+    rec = (C.c_int * max(n_records, 1))()
+    _check(load().hero_attention_bf16_static_status(_stream(), C.byref(gave_up), rec if n_records else None, n_records),
+           "hero_attention_bf16_static_status")
+    return gave_up.value, list(rec)[:n_records]
+
+
 def hero_isolated_status():
     _check(load().hero_isolated_status(_stream()), "hero_isolated_status")
+
+
+def hero_selftest_wait_timeout(budget_us: int = 50):
+    """Make one bounded device-side wait run out on purpose (raises the isolated calls' status word)."""
+    _require_cuda()
+    _check(load().hero_selftest_wait_timeout(None, budget_us, _stream()), "hero_selftest_wait_timeout")
+
+
+def hero_gather_ln_modulate(x, add, idx, shift, scale, out):
+    """out[b, i] = LN(x[b, idx[i]] (+ add[b, idx[i]])) * (1 + scale[b]) + shift[b]; shift/scale fp32 [B, D]."""
+    _require_cuda()
+    B, N, D = x.shape
+    n_sel = out.shape[1]
+    assert shift.dtype == torch.float32 and scale.dtype == torch.float32 and shift.stride(0) == scale.stride(0)
+    _check(load().hero_gather_ln_modulate(_ptr(x), _ptr(add), _ptr(idx), _ptr(shift), _ptr(scale), shift.stride(0),
+                                          _ptr(out), B, N, n_sel, D, dtype_code(x.dtype), _stream()),
+           "hero_gather_ln_modulate")
+    return out
 
 
 def device_weights(host_weights: dict, dtype, device="cuda") -> dict:

@@ -28,7 +28,10 @@ struct BlockMem {
   uint16_t* ages[2] = {nullptr, nullptr};                // shallow: double-buffered age counters
   int ages_cur = 0;
   int calls = 0;              // selections made on this block
+  unsigned filled = 0;        // shallow: which of K, V, G_attn, G_ffn hold valid rows (bits 0..3); a full pass
+                              // sets all four, planting a cache through hero_state_set sets its bit
 };
+constexpr unsigned kAllCaches = 0xFu;
 
 }  // namespace hero
 
@@ -67,7 +70,8 @@ struct hero_ctx {
   void *ws_a = nullptr, *ws_q = nullptr, *ws_o = nullptr, *ws_u = nullptr;
   float* mod = nullptr;                  // [n_blocks, B, n_mod*D] adaLN vectors, one slot per block
   int* idx_ws = nullptr;                 // [n_shallow, idx_cap] selection lists of the current step
-  int* d_status = nullptr;
+  int* d_status = nullptr;                // word 0: kernels that gave up on a wait; then one word per attention CTA
+  int status_ctas = 0;
   void *x_stage = nullptr, *temb_stage = nullptr;
   int n_full = 0, s_prev = 0, s_last = 0;
   int mode1_n_sel = 0;
@@ -167,7 +171,7 @@ int run_attention(hero_ctx* c, const void* q, const void* k, const void* v, void
   const hero_config& g = c->cfg;
   LaunchScope scope(c, HERO_PROF_ATTENTION);
   if (g.dtype == HERO_DTYPE_BF16)
-    return launch_tc_attention(q, k, v, o, g.batch, n_q, c->N, g.n_heads, c->d_status, c->stream);
+    return launch_tc_attention(q, k, v, o, g.batch, n_q, c->N, g.n_heads, c->d_status, c->status_ctas, c->stream);
   return launch_simt_attention(q, k, v, o, g.batch, n_q, c->N, g.n_heads, g.head_dim, g.dtype, c->stream);
 }
 
@@ -260,7 +264,7 @@ int refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, const i
     LaunchScope scope(c, HERO_PROF_ATTENTION);
     if (g.dtype == HERO_DTYPE_BF16)
       HERO_TRY(launch_tc_attention(c->ws_q, c->kv_cmp[0], c->kv_cmp[1], c->ws_o, B, n_sel, n_att, g.n_heads, c->d_status,
-                                   c->stream));
+                                   c->status_ctas, c->stream));
     else
       HERO_TRY(launch_simt_attention(c->ws_q, c->kv_cmp[0], c->kv_cmp[1], c->ws_o, B, n_sel, n_att, g.n_heads, g.head_dim,
                                      g.dtype, c->stream));
@@ -304,6 +308,7 @@ int refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, const i
       bm.last_slot = new_slot;
       if (bm.n_hist < 2) bm.n_hist++;
     } else {
+      bm.filled = kAllCaches;
       HERO_CUDA_TRY(cudaMemsetAsync(bm.ages[bm.ages_cur], 0, (size_t)c->n_video * sizeof(uint16_t), c->stream));
     }
   }
@@ -368,11 +373,20 @@ int validate(const hero_config* g) {
   if ((g->qk_norm != 0 && g->qk_norm != 1) || (g->rope != 0 && g->rope != 1)) return HERO_ERR_ARG;
   if ((g->qk_norm || g->rope) && (g->head_dim % 2 != 0 || g->head_dim > 256)) return HERO_ERR_ARG;
   if (g->dtype == HERO_DTYPE_BF16) {
-    if (g->head_dim != 64 || g->hidden % 8 || g->ffn_dim % 8 || g->temb_dim % 8) return HERO_ERR_ALIGN;
+    // the tensor-core GEMM cuts its output into 32-column pieces per destination (q | k | v, FFN width)
+    if (g->head_dim != 64 || g->hidden % 32 || g->ffn_dim % 32 || g->temb_dim % 8) return HERO_ERR_ALIGN;
   } else {
     if (g->head_dim != 32 && g->head_dim != 64 && g->head_dim != 128) return HERO_ERR_ARG;
     if (g->hidden % 4 || g->ffn_dim % 4 || g->temb_dim % 4) return HERO_ERR_ALIGN;
   }
+  // dynamic shared memory the streaming kernels take without an opt-in (48 KB): SiLU(temb) of the whole batch
+  // in the adaLN kernels, one fp32 row in the generic LayerNorm prologue (the bf16 warp-per-row kernel, used
+  // for hidden = 1024 / 2048 / 3072 / 4096, needs none)
+  constexpr long long kPlainSmem = 48 * 1024;
+  if ((long long)g->batch * g->temb_dim * 4 > kPlainSmem) return HERO_ERR_ARG;
+  const bool warp_ln = g->dtype == HERO_DTYPE_BF16 &&
+                       (g->hidden == 1024 || g->hidden == 2048 || g->hidden == 3072 || g->hidden == 4096);
+  if (!warp_ln && (long long)g->hidden * 4 > kPlainSmem) return HERO_ERR_ARG;
   const long long n_video = (long long)g->frames * g->grid_h * g->grid_w;
   if (n_video + g->n_text > (1ll << 30)) return HERO_ERR_ARG;
   return HERO_OK;
@@ -483,7 +497,9 @@ int hero_init(hero_ctx** out, const hero_config* cfg, const hero_block_weights* 
   A(&c->ws_u, (size_t)cfg->batch * c->N * cfg->ffn_dim * c->esz);
   A((void**)&c->mod, (size_t)cfg->n_blocks * cfg->batch * c->n_mod * cfg->hidden * sizeof(float));
   A((void**)&c->idx_ws, (size_t)(cfg->n_shallow > 0 ? cfg->n_shallow : 1) * c->idx_cap * sizeof(int));
-  A((void**)&c->d_status, 16);
+  // the largest attention launch of this context is the full pass (n_q = N)
+  c->status_ctas = cfg->dtype == HERO_DTYPE_BF16 ? (int)tc_attention_grid(cfg->batch, c->N, cfg->n_heads) : 0;
+  A((void**)&c->d_status, (size_t)(4 + c->status_ctas) * sizeof(int));
   A(&c->x_stage, tensor);
   A(&c->temb_stage, (size_t)cfg->batch * cfg->temb_dim * c->esz);
   if (rc != HERO_OK) { hero_destroy(c); return rc; }
@@ -491,7 +507,7 @@ int hero_init(hero_ctx** out, const hero_config* cfg, const hero_block_weights* 
     cudaError_t er = cudaMemcpy(c->rope_tab, rope_host.data(), rope_host.size() * sizeof(float2), cudaMemcpyHostToDevice);
     if (er != cudaSuccess) { set_cuda_error(er, "cudaMemcpy(rope table)"); hero_destroy(c); return HERO_ERR_CUDA; }
   }
-  cudaError_t e = cudaMemsetAsync(c->d_status, 0, 16, c->stream);
+  cudaError_t e = cudaMemsetAsync(c->d_status, 0, (size_t)(4 + c->status_ctas) * sizeof(int), c->stream);
   if (e != cudaSuccess) { set_cuda_error(e, "cudaMemsetAsync"); hero_destroy(c); return HERO_ERR_CUDA; }
   rc = hero_reset(c);
   if (rc != HERO_OK) { hero_destroy(c); return rc; }
@@ -503,7 +519,7 @@ int hero_reset(hero_ctx* c) {
   if (!c) return HERO_ERR_ARG;
   for (int l = 0; l < c->cfg.n_blocks; ++l) {
     BlockMem& bm = c->blk[l];
-    bm.calls = 0; bm.ages_cur = 0; bm.n_hist = 0; bm.last_slot = 0;
+    bm.calls = 0; bm.ages_cur = 0; bm.n_hist = 0; bm.last_slot = 0; bm.filled = 0;
     if (bm.ages[0]) HERO_CUDA_TRY(cudaMemsetAsync(bm.ages[0], 0, (size_t)c->n_video * 2, c->stream));
     if (bm.ages[1]) HERO_CUDA_TRY(cudaMemsetAsync(bm.ages[1], 0, (size_t)c->n_video * 2, c->stream));
   }
@@ -547,11 +563,11 @@ int hero_profile_end(hero_ctx* c, double* ms, long long* launches) {
 
 int hero_check_status(hero_ctx* c) {
   if (!c) return HERO_ERR_ARG;
-  int st[4] = {0, 0, 0, 0};
-  HERO_CUDA_TRY(cudaMemcpyAsync(st, c->d_status, 16, cudaMemcpyDeviceToHost, c->stream));
+  int st = 0;
+  HERO_CUDA_TRY(cudaMemcpyAsync(&st, c->d_status, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
   HERO_CUDA_TRY(cudaStreamSynchronize(c->stream));
-  if (st[0] != 0) {
-    cudaMemsetAsync(c->d_status, 0, 16, c->stream);
+  if (st != 0) {
+    cudaMemsetAsync(c->d_status, 0, sizeof(int), c->stream);
     return HERO_ERR_TIMEOUT;
   }
   return HERO_OK;
@@ -587,6 +603,7 @@ int hero_refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, co
   if (n_sel == 0) {                                        // empty list: nothing refreshed,
     if (block >= c->cfg.n_shallow) return HERO_ERR_ARG;    // the residual adds still happen
     BlockMem& bm = c->blk[block];
+    if (bm.filled != kAllCaches) return HERO_ERR_STATE;    // nothing cached yet to add
     HERO_LAUNCH(c, HERO_PROF_RESIDUAL, launch_residual2(d_x, bm.g[0], bm.g[1], c->elems, c->cfg.dtype, c->stream));
     return HERO_OK;
   }
@@ -596,6 +613,8 @@ int hero_refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, co
   } else {
     if (n_sel < 0 || n_sel > c->N) return HERO_ERR_ARG;
     if (block >= c->cfg.n_shallow) return HERO_ERR_ARG;   // deep blocks keep no K/V cache to refresh against
+    // a partial refresh merges with the cache (Eq. 3): the block must have seen a full pass first
+    if (c->blk[block].filled != kAllCaches) return HERO_ERR_STATE;
   }
   return refresh_block(c, block, d_x, d_temb, d_idx, n_sel);
 }
@@ -782,14 +801,40 @@ int hero_scatter_rows(const void* src, const int* idx, void* dst, int B, int N, 
   return launch_scatter_rows(src, idx, dst, B, N, n_sel, D, dtype, (cudaStream_t)stream);
 }
 
+// Eq. 2's prologue alone: out[b, i, :] = LN(x[b, idx[i], :] (+ add[b, idx[i], :])) * (1 + scale[b, :]) + shift[b, :]
+int hero_gather_ln_modulate(const void* d_x, const void* d_add, const int* d_idx, const float* d_shift,
+                            const float* d_scale, int mod_ld, void* d_out, int B, int N, int n_sel, int D, int dtype,
+                            void* stream) {
+  if (B < 0 || N < 0 || n_sel < 0 || n_sel > N || D <= 0 || mod_ld < D) return HERO_ERR_ARG;
+  if (dtype != HERO_DTYPE_FP32 && dtype != HERO_DTYPE_BF16) return HERO_ERR_ARG;
+  if (B == 0 || n_sel == 0) return HERO_OK;
+  if (!d_x || !d_shift || !d_scale || !d_out) return HERO_ERR_ARG;
+  if (!aligned16(d_x) || !aligned16(d_out) || (d_add && !aligned16(d_add))) return HERO_ERR_ALIGN;
+  if (D % (dtype == HERO_DTYPE_BF16 ? 8 : 4)) return HERO_ERR_ALIGN;
+  const bool warp_ln = dtype == HERO_DTYPE_BF16 && (D == 1024 || D == 2048 || D == 3072 || D == 4096);
+  if (!warp_ln && (long long)D * 4 > 48 * 1024) return HERO_ERR_ARG;      // one fp32 row of shared memory
+  return launch_gather_ln_modulate(d_x, d_add, d_idx, d_shift, d_scale, mod_ld, d_out, B, N, n_sel, D, 1e-5f, dtype,
+                                   (cudaStream_t)stream);
+}
+
 // The isolated tensor-core calls own a status word each; a timeout is reported on the next call.
+// The words live in the memory of the device that is current at the call (one set per device, kept until exit):
+// word 0 for give-ups, then one word per attention CTA (larger grids run the safe attention kernel alone).
+constexpr int kIsolatedStatusCtas = 65536;
 static int* isolated_status() {
-  static int* p = nullptr;
-  if (!p) {
-    if (cudaMalloc((void**)&p, 16) != cudaSuccess) { p = nullptr; return nullptr; }
-    cudaMemset(p, 0, 16);
-  }
-  return p;
+  static PerDeviceOnce once;
+  static int* word[kMaxDevices];
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  const int rc = per_device_once(once, [](int d) {
+    int* p = nullptr;
+    const size_t bytes = (size_t)(4 + kIsolatedStatusCtas) * sizeof(int);
+    if (cudaMalloc((void**)&p, bytes) != cudaSuccess) { cudaGetLastError(); return HERO_ERR_NOMEM; }
+    if (cudaMemset(p, 0, bytes) != cudaSuccess) { cudaFree(p); return HERO_ERR_CUDA; }
+    word[d] = p;
+    return HERO_OK;
+  });
+  return rc == HERO_OK ? word[dev] : nullptr;
 }
 static int poll_isolated_status(cudaStream_t s) {
   int* p = isolated_status();
@@ -797,7 +842,7 @@ static int poll_isolated_status(cudaStream_t s) {
   int st = 0;
   HERO_CUDA_TRY(cudaMemcpyAsync(&st, p, 4, cudaMemcpyDeviceToHost, s));
   HERO_CUDA_TRY(cudaStreamSynchronize(s));
-  if (st) { cudaMemset(p, 0, 16); return HERO_ERR_TIMEOUT; }
+  if (st) { cudaMemset(p, 0, sizeof(int)); return HERO_ERR_TIMEOUT; }
   return HERO_OK;
 }
 
@@ -821,11 +866,33 @@ int hero_attention_bf16(const void* q, const void* k, const void* v, void* o, in
   if (!q || !k || !v || !o) return HERO_ERR_ARG;
   int* st = isolated_status();
   if (!st) return HERO_ERR_NOMEM;
-  return launch_tc_attention(q, k, v, o, B, n_q, N, heads, st, (cudaStream_t)stream);
+  return launch_tc_attention(q, k, v, o, B, n_q, N, heads, st, kIsolatedStatusCtas, (cudaStream_t)stream);
+}
+
+int hero_attention_bf16_safe(const void* q, const void* k, const void* v, void* o, int B, int n_q, int N, int heads,
+                             void* stream) {
+  if (B < 0 || n_q < 0 || N <= 0 || heads <= 0) return HERO_ERR_ARG;
+  if (B == 0 || n_q == 0) return HERO_OK;
+  if (!q || !k || !v || !o) return HERO_ERR_ARG;
+  int* st = isolated_status();
+  if (!st) return HERO_ERR_NOMEM;
+  return launch_tc_attention_safe(q, k, v, o, B, n_q, N, heads, st, (cudaStream_t)stream);
 }
 
 // Synchronise `stream` and report whether an isolated tensor-core call gave up on a wait.
 int hero_isolated_status(void* stream) { return poll_isolated_status((cudaStream_t)stream); }
+
+// Self-test of the give-up path: one thread block waits, with a budget of `budget_us` microseconds, on a
+// barrier that nobody will ever complete, through the same bounded-wait helper the tensor-core kernels use;
+// the wait runs out, the block raises the status word and returns.  With a context the word is the
+// context's (hero_check_status then reports HERO_ERR_TIMEOUT once), without one it is the word of the
+// isolated tensor-core calls (hero_isolated_status reports it).
+int hero_selftest_wait_timeout(hero_ctx* c, int budget_us, void* stream) {
+  if (budget_us < 1 || budget_us > 100000) return HERO_ERR_ARG;
+  int* st = c ? c->d_status : isolated_status();
+  if (!st) return HERO_ERR_NOMEM;
+  return launch_wait_timeout_selftest(st, budget_us, c ? c->stream : (cudaStream_t)stream);
+}
 
 // ---------------------------------------------------------------- state access
 static int state_ptr(hero_ctx* c, int block, int what, void** p, size_t* bytes) {
@@ -883,6 +950,12 @@ int hero_state_set(hero_ctx* c, int block, int what, const void* h_in, long long
   HERO_CUDA_TRY(cudaStreamSynchronize(c->stream));
   if (what == HERO_STATE_STACK_LAST) { if (c->stack_n < 1) c->stack_n = 1; return HERO_OK; }
   if (what == HERO_STATE_STACK_PREV) { c->stack_n = 2; return HERO_OK; }
+  if (block < c->cfg.n_shallow) {    // planting a shallow block's cache marks it as valid
+    if (what == HERO_STATE_K) c->blk[block].filled |= 1u;
+    if (what == HERO_STATE_V) c->blk[block].filled |= 2u;
+    if (what == HERO_STATE_G_ATTN) c->blk[block].filled |= 4u;
+    if (what == HERO_STATE_G_FFN) c->blk[block].filled |= 8u;
+  }
   if (block >= c->cfg.n_shallow) {   // planting a deep block's history marks the slots as valid
     BlockMem& bm = c->blk[block];
     if (what == HERO_STATE_G_ATTN || what == HERO_STATE_G_FFN) { if (bm.n_hist < 1) bm.n_hist = 1; }

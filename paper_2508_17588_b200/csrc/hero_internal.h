@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "hero.h"
 
 namespace hero {
@@ -29,6 +31,30 @@ void set_cuda_error(cudaError_t e, const char* what);
   } while (0)
 
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ---------------------------------------------------------------------------
+// Set-up that has to happen once PER DEVICE (a kernel's shared-memory opt-in, a status word in that
+// device's memory, its SM count): a process may drive several GPUs, so nothing of this kind may be
+// cached per process.  `fn` runs under the table's lock, with the calling thread's device current, the
+// first time that device comes by; a failure is not remembered and is retried on the next call.
+// ---------------------------------------------------------------------------
+constexpr int kMaxDevices = 64;
+struct PerDeviceOnce {
+  std::mutex mu;
+  bool done[kMaxDevices] = {};
+};
+template <class F>
+int per_device_once(PerDeviceOnce& once, F&& fn) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return HERO_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(once.mu);
+  if (!once.done[dev]) {
+    const int rc = fn(dev);
+    if (rc != HERO_OK) return rc;
+    once.done[dev] = true;
+  }
+  return HERO_OK;
+}
 static inline size_t dtype_size(int dtype) { return dtype == HERO_DTYPE_BF16 ? 2 : 4; }
 
 // ---------------------------------------------------------------------------
@@ -140,8 +166,15 @@ int launch_simt_attention(const void* q, const void* k, const void* v, void* o, 
 int tc_init_driver_api();   // resolves cuTensorMapEncodeTiled once
 int launch_tc_gemm(const void* a, const void* w, const void* bias, int M, int Nout, int K,
                    const GemmOut& out, int* d_status, cudaStream_t s);
+// d_status: word 0 (give-up counter) followed by status_ctas per-CTA words
 int launch_tc_attention(const void* q, const void* k, const void* v, void* o, int B, int n_q, int N,
-                        int heads, int* d_status, cudaStream_t s);
+                        int heads, int* d_status, int status_ctas, cudaStream_t s);
+int launch_tc_attention_safe(const void* q, const void* k, const void* v, void* o, int B, int n_q, int N,
+                             int heads, int* d_status, cudaStream_t s);
+long long tc_attention_grid(int B, int n_q, int heads);   // CTAs of one attention launch
+
+// one thread block, no TMA, no TMEM: a bounded wait on a barrier nobody arms; raises *d_status and returns
+int launch_wait_timeout_selftest(int* d_status, int budget_us, cudaStream_t s);
 
 int num_sms();
 

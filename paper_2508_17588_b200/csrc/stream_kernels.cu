@@ -6,14 +6,19 @@
 
 namespace hero {
 
+// SM count of the calling thread's current device (looked up once per device).
 int num_sms() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-  }
-  return n;
+  static PerDeviceOnce once;
+  static int count[kMaxDevices];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 148;
+  per_device_once(once, [](int d) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, d) != cudaSuccess || n <= 0) n = 148;
+    count[d] = n;
+    return HERO_OK;
+  });
+  return count[dev] > 0 ? count[dev] : 148;
 }
 
 namespace {
@@ -520,79 +525,99 @@ gather_ln_modulate_kernel(const T* __restrict__ x, const T* __restrict__ add, co
 }
 
 // bf16 rows of 256 * VPL elements: one WARP per refreshed row, the row held in registers (VPL
-// 16-byte packets per lane), statistics by warp shuffles alone - no shared memory, no block barrier,
-// 8 independent rows in flight per CTA.
+// 16-byte packets per lane), statistics by warp shuffles alone - no block barrier per row, 8 independent
+// rows in flight per CTA.  The CTAs are persistent and each serves ONE batch item: it first puts that
+// item's (1 + scale) and shift vectors into shared memory in fp32 (24 KB at D = 3072, once per CTA), so a
+// row costs its own 6 KB in and 6 KB out of HBM plus shared-memory reads - not 24 KB of L1/L2 traffic for
+// the vectors again.  Layout of the vectors: four planes of float4, [low/high half of a packet's (1 + scale),
+// low/high half of its shift][packet], so that the lanes of a warp read consecutive 16-byte words.
 template <int VPL>
 __global__ void __launch_bounds__(256, (VPL > 12) ? 1 : 2)
 gather_ln_modulate_warp_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ add,
                                const int* __restrict__ idx, const float* __restrict__ shift,
                                const float* __restrict__ scale, int mod_ld, __nv_bfloat16* __restrict__ a, int N,
-                               int n_sel, long long rows, float eps) {
+                               int n_sel, int B, float eps) {
   using V = Vec<__nv_bfloat16>;
-  constexpr int D = VPL * 256;
-  const int lane = threadIdx.x & 31;
-  const long long m = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
-  if (m >= rows) return;
-  const int b = (int)(m / n_sel), i = (int)(m - (long long)b * n_sel);
-  const long long row = (long long)b * N + (idx ? __ldg(idx + i) : i);
-  const V* xr = reinterpret_cast<const V*>(x + row * D);
-  V raw[VPL];
-#pragma unroll
-  for (int c = 0; c < VPL; ++c) raw[c].raw = __ldcs(&xr[c * 32 + lane].raw);
-  float f[VPL][8];
-#pragma unroll
-  for (int c = 0; c < VPL; ++c) raw[c].unpack(f[c]);
-  if (add) {
-    const V* ar = reinterpret_cast<const V*>(add + row * D);
-#pragma unroll
-    for (int c = 0; c < VPL; ++c) raw[c].raw = __ldcs(&ar[c * 32 + lane].raw);
-#pragma unroll
-    for (int c = 0; c < VPL; ++c) {
-      float g[8];
-      raw[c].unpack(g);
-#pragma unroll
-      for (int q = 0; q < 8; ++q) f[c][q] += g[q];
+  constexpr int D = VPL * 256, kPackets = VPL * 32;
+  extern __shared__ float4 s_mod[];                 // [4][kPackets]
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int b = blockIdx.x % B, slot = blockIdx.x / B, slots = gridDim.x / B;
+  {
+    const float4* sc = reinterpret_cast<const float4*>(scale + (long long)b * mod_ld);
+    const float4* sh = reinterpret_cast<const float4*>(shift + (long long)b * mod_ld);
+    for (int i = threadIdx.x; i < 2 * kPackets; i += 256) {        // float4 i covers columns [4i, 4i + 4)
+      const float4 s4 = __ldg(sc + i), h4 = __ldg(sh + i);
+      s_mod[(i & 1) * kPackets + (i >> 1)] = make_float4(1.0f + s4.x, 1.0f + s4.y, 1.0f + s4.z, 1.0f + s4.w);
+      s_mod[(2 + (i & 1)) * kPackets + (i >> 1)] = h4;
     }
   }
-  float sum = 0.f;
+  __syncthreads();
+  for (int i = slot * 8 + warp; i < n_sel; i += slots * 8) {
+    const long long row = (long long)b * N + (idx ? __ldg(idx + i) : i);
+    const V* xr = reinterpret_cast<const V*>(x + row * D);
+    V raw[VPL];
 #pragma unroll
-  for (int c = 0; c < VPL; ++c)
+    for (int c = 0; c < VPL; ++c) raw[c].raw = __ldcs(&xr[c * 32 + lane].raw);
+    float f[VPL][8];
 #pragma unroll
-    for (int q = 0; q < 8; ++q) sum += f[c][q];
+    for (int c = 0; c < VPL; ++c) raw[c].unpack(f[c]);
+    if (add) {
+      const V* ar = reinterpret_cast<const V*>(add + row * D);
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
-  const float mean = sum / (float)D;
-  float sq = 0.f;
+      for (int c = 0; c < VPL; ++c) raw[c].raw = __ldcs(&ar[c * 32 + lane].raw);
 #pragma unroll
-  for (int c = 0; c < VPL; ++c)
+      for (int c = 0; c < VPL; ++c) {
+        float g[8];
+        raw[c].unpack(g);
 #pragma unroll
-    for (int q = 0; q < 8; ++q) { const float d = f[c][q] - mean; sq = fmaf(d, d, sq); }
+        for (int q = 0; q < 8; ++q) f[c][q] += g[q];
+      }
+    }
+    float sum = 0.f;
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xFFFFFFFFu, sq, o);
-  const float rstd = 1.0f / sqrtf(sq / (float)D + eps);
-  const float4* sh = reinterpret_cast<const float4*>(shift + (long long)b * mod_ld);
-  const float4* sc = reinterpret_cast<const float4*>(scale + (long long)b * mod_ld);
-  V* out = reinterpret_cast<V*>(a + m * D);
+    for (int c = 0; c < VPL; ++c)
 #pragma unroll
-  for (int c = 0; c < VPL; ++c) {
-    const int v = c * 32 + lane;       // packet index: columns [8v, 8v + 8)
-    const float4 s0 = __ldg(sc + 2 * v), s1 = __ldg(sc + 2 * v + 1), h0 = __ldg(sh + 2 * v), h1 = __ldg(sh + 2 * v + 1);
-    const float scl[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
-    const float sft[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
-    float r[8];
+      for (int q = 0; q < 8; ++q) sum += f[c][q];
 #pragma unroll
-    for (int q = 0; q < 8; ++q) r[q] = fmaf((f[c][q] - mean) * rstd, 1.0f + scl[q], sft[q]);
-    V o; o.pack(r);
-    out[v] = o;
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+    const float mean = sum / (float)D;
+    float sq = 0.f;
+#pragma unroll
+    for (int c = 0; c < VPL; ++c)
+#pragma unroll
+      for (int q = 0; q < 8; ++q) { const float d = f[c][q] - mean; sq = fmaf(d, d, sq); }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xFFFFFFFFu, sq, o);
+    const float rstd = 1.0f / sqrtf(sq / (float)D + eps);
+    V* out = reinterpret_cast<V*>(a + ((long long)b * n_sel + i) * D);
+#pragma unroll
+    for (int c = 0; c < VPL; ++c) {
+      const int v = c * 32 + lane;       // packet index: columns [8v, 8v + 8)
+      const float4 s0 = s_mod[v], s1 = s_mod[kPackets + v], h0 = s_mod[2 * kPackets + v], h1 = s_mod[3 * kPackets + v];
+      const float scl[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+      const float sft[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
+      float r[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) r[q] = fmaf((f[c][q] - mean) * rstd, scl[q], sft[q]);
+      V o; o.pack(r);
+      __stcs(&out[v].raw, o.raw);
+    }
   }
 }
 
 template <int VPL>
 int gather_ln_warp(const void* x, const void* add, const int* idx, const float* shift, const float* scale, int mod_ld,
-                   void* a, int N, int n_sel, long long rows, float eps, cudaStream_t s) {
+                   void* a, int N, int n_sel, int B, float eps, cudaStream_t s) {
   using T = __nv_bfloat16;
-  gather_ln_modulate_warp_kernel<VPL><<<(unsigned)((rows + 7) / 8), 256, 0, s>>>(
-      (const T*)x, (const T*)add, idx, shift, scale, mod_ld, (T*)a, N, n_sel, rows, eps);
+  // persistent CTAs, the same number for every batch item; two per SM (one for the widest rows) is all that fits
+  const int per_sm = VPL > 12 ? 1 : 2;
+  int slots = (num_sms() * per_sm + B - 1) / B;
+  const int need = (n_sel + 7) / 8;
+  if (slots > need) slots = need;
+  if (slots < 1) slots = 1;
+  const size_t smem = (size_t)4 * VPL * 32 * sizeof(float4);
+  gather_ln_modulate_warp_kernel<VPL><<<(unsigned)(slots * B), 256, smem, s>>>(
+      (const T*)x, (const T*)add, idx, shift, scale, mod_ld, (T*)a, N, n_sel, B, eps);
   HERO_CUDA_TRY(cudaGetLastError());
   return HERO_OK;
 }
@@ -786,10 +811,10 @@ int launch_gather_ln_modulate(const void* x, const void* add, const int* idx, co
     if (D % 8) return HERO_ERR_ALIGN;
     // the adaLN vectors are read as float4: every block's slice starts 16-byte aligned when mod_ld % 4 == 0
     const bool vec_ok = mod_ld % 4 == 0 && ((reinterpret_cast<uintptr_t>(shift) | reinterpret_cast<uintptr_t>(scale)) & 15) == 0;
-    if (vec_ok && D == 1024) return gather_ln_warp<4>(x, add, idx, shift, scale, mod_ld, a, N, n_sel, rows, eps, s);
-    if (vec_ok && D == 2048) return gather_ln_warp<8>(x, add, idx, shift, scale, mod_ld, a, N, n_sel, rows, eps, s);
-    if (vec_ok && D == 3072) return gather_ln_warp<12>(x, add, idx, shift, scale, mod_ld, a, N, n_sel, rows, eps, s);
-    if (vec_ok && D == 4096) return gather_ln_warp<16>(x, add, idx, shift, scale, mod_ld, a, N, n_sel, rows, eps, s);
+    if (vec_ok && D == 1024) return gather_ln_warp<4>(x, add, idx, shift, scale, mod_ld, a, N, n_sel, B, eps, s);
+    if (vec_ok && D == 2048) return gather_ln_warp<8>(x, add, idx, shift, scale, mod_ld, a, N, n_sel, B, eps, s);
+    if (vec_ok && D == 3072) return gather_ln_warp<12>(x, add, idx, shift, scale, mod_ld, a, N, n_sel, B, eps, s);
+    if (vec_ok && D == 4096) return gather_ln_warp<16>(x, add, idx, shift, scale, mod_ld, a, N, n_sel, B, eps, s);
     gather_ln_modulate_kernel<T><<<(unsigned)rows, kLnThreads, smem, s>>>((const T*)x, (const T*)add, idx, shift,
                                                                            scale, mod_ld, (T*)a, N, n_sel, D, eps);
   } else {

@@ -52,29 +52,39 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                    uint64_t budget_ns) {
   const uint64_t t0 = global_timer_ns();
   for (uint32_t it = 0; it < kWaitMaxPolls; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if ((it & 63u) == 63u && global_timer_ns() - t0 > kWaitBudgetNs) break;
+    if ((it & 63u) == 63u && global_timer_ns() - t0 > budget_ns) break;
     __nanosleep(64);
   }
   *abort_flag = 1;
   return false;
 }
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          uint64_t budget_ns = kWaitBudgetNs) {
   for (uint32_t it = 0; it < kWaitFastPolls; ++it)
     if (mbar_try_wait(bar, parity)) return true;
-  return mbar_wait_slow(bar, parity, abort_flag);
+  return mbar_wait_slow(bar, parity, abort_flag, budget_ns);
 }
-// The same wait for a whole converged warp whose lanes all poll the same barrier: one poll is one
-// warp-wide instruction, so the fast path is uniform by construction and only the slow path (where a lane
-// might give up a poll earlier than another) pays for a vote.
-__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t it = 0; it < kWaitFastPolls; ++it)
-    if (mbar_try_wait(bar, parity)) return true;
-  return __all_sync(0xFFFFFFFFu, mbar_wait_slow(bar, parity, abort_flag));
+// The same wait for a whole warp whose lanes all poll the same barrier.  The lanes are brought together
+// first (a barrier among the lanes, not a vote), so that every lane enters the poll loop in the same
+// instruction: one poll is then one warp-wide instruction with one answer, the fast path is uniform, and
+// the vote at the end of the slow path always finds all 32 lanes - no lane can have left through the fast
+// path while the others wait for it in the vote.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                               uint64_t budget_ns = kWaitBudgetNs) {
+  __syncwarp();
+  bool done = false;
+  for (uint32_t it = 0; it < kWaitFastPolls && !done; ++it) done = mbar_try_wait(bar, parity);
+  // a completed phase stays completed, so lanes that saw it early and lanes that saw it late agree once all
+  // have seen it; the vote makes the exit itself warp-uniform
+  if (__all_sync(0xFFFFFFFFu, done)) return true;
+  if (!done) done = mbar_wait_slow(bar, parity, abort_flag, budget_ns);
+  return __all_sync(0xFFFFFFFFu, done);
 }
 
 // ---------------------------------------------------------------- TMA (no multicast anywhere)
@@ -169,6 +179,25 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
       "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
       "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr), "r"(r[0]),
+               "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+               : "memory");
+}
+// One lane of a converged warp, the same one every time for a full mask.  Code that all lanes run and only
+// the elected lane acts on keeps its loop counters and operands warp-uniform, which is what lets the compiler
+// feed the tensor-core instructions from uniform registers.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t"
+      "}"
+      : "=r"(pred));
+  return pred != 0;
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 

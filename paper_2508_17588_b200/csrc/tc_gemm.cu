@@ -163,28 +163,34 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // All 32 lanes run the loop and one elected lane issues: tile counters, stage addresses and descriptors
+    // then stay warp-uniform values instead of one diverged lane's private registers, which is what the
+    // tensor-core instructions are fed from.
+    {
+      const bool leader = elect_one();
       constexpr uint32_t idesc = idesc_bf16(kBM, kBN, 0);
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
       int t = 0;
       for (int tile = blockIdx.x; tile < n_tiles_total && ok; tile += gridDim.x, ++t) {
         const int acc = t & 1;
-        if (!(ok = mbar_wait(&acc_empty[acc], ((t >> 1) & 1) ^ 1, abort_flag))) break;
+        if (!(ok = mbar_wait_warp(&acc_empty[acc], ((t >> 1) & 1) ^ 1, abort_flag))) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)acc * kBN;
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!(ok = mbar_wait(&full[stage], phase, abort_flag))) break;
+          if (!(ok = mbar_wait_warp(&full[stage], phase, abort_flag))) break;
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + (size_t)stage * kStageBytes);
           const uint64_t da = smem_desc_sw128(sa, 1024), db = smem_desc_sw128(sa + kABytes, 1024);
+          if (leader) {
 #pragma unroll
-          for (int k = 0; k < kBK / 16; ++k)   // +32 bytes (encoded >>4) per K step of 16 inside the swizzle atom
-            mma_ss(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
-          mma_commit(&empty[stage]);
+            for (int k = 0; k < kBK / 16; ++k)   // +32 bytes (encoded >>4) per K step of 16 inside the swizzle atom
+              mma_ss(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+            mma_commit(&empty[stage]);
+          }
           if (++stage == kStages) { stage = 0; phase ^= 1; }
         }
-        if (ok) mma_commit(&acc_full[acc]);
+        if (ok && leader) mma_commit(&acc_full[acc]);
       }
     }
   } else {
@@ -252,7 +258,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, kTmemCols); }
 }
 
+// Self-test of the bounded wait: the barrier below is initialised for one arrival that never comes.
+__global__ void wait_timeout_selftest_kernel(int* __restrict__ status, unsigned long long budget_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) { mbar_init(&bar, 1); abort_flag = 0; mbar_fence_init(); }
+  __syncthreads();
+  const bool ok = mbar_wait_warp(&bar, 0, &abort_flag, budget_ns);
+  __syncthreads();
+  if (threadIdx.x == 0 && (!ok || abort_flag)) atomicExch(status, 1);
+}
+
 }  // namespace
+
+int launch_wait_timeout_selftest(int* d_status, int budget_us, cudaStream_t s) {
+  wait_timeout_selftest_kernel<<<1, 64, 0, s>>>(d_status, (unsigned long long)budget_us * 1000ull);
+  HERO_CUDA_TRY(cudaGetLastError());
+  return HERO_OK;
+}
 
 int launch_tc_gemm(const void* a, const void* w, const void* bias, int M, int Nout, int K, const GemmOut& out,
                    int* d_status, cudaStream_t s) {
@@ -274,12 +297,11 @@ int launch_tc_gemm(const void* a, const void* w, const void* bias, int M, int No
     const uint32_t box[2] = {(uint32_t)kBK, (uint32_t)kBN};
     HERO_TRY(make_tmap_bf16(&tm_w, w, 2, dims, str, box));
   }
-  static std::once_flag attr_once;
-  static cudaError_t attr_err = cudaSuccess;
-  std::call_once(attr_once, [] {
-    attr_err = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem);
-  });
-  HERO_CUDA_TRY(attr_err);
+  static PerDeviceOnce attr_once;            // the opt-in is a property of the kernel ON a device
+  HERO_TRY(per_device_once(attr_once, [](int) {
+    HERO_CUDA_TRY(cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem));
+    return HERO_OK;
+  }));
   const int tiles = ((M + kBM - 1) / kBM) * ((Nout + kBN - 1) / kBN);
   const int grid = tiles < num_sms() ? tiles : num_sms();
   tc_gemm_kernel<<<grid, kGemmThreads, kGemmSmem, s>>>(tm_a, tm_w, (const __nv_bfloat16*)bias, out, M, Nout, K,

@@ -169,6 +169,8 @@ def test_call_order_and_argument_errors_with_a_live_context():
         return e.value.code
 
     assert code(lambda: hero.hero_step(2, x, t)) == -4                                  # cached step before any full step
+    assert code(lambda: hero.hero_refresh_block(0, x, t, idx, 4)) == -4                 # partial refresh before any full pass
+    assert code(lambda: hero.hero_refresh_block(0, x, t, idx, 0)) == -4                 # nothing cached yet to add either
     assert code(lambda: hero.hero_extrapolate_block(2, x, 1, 1)) == -4                  # no history yet
     assert code(lambda: hero.hero_extrapolate_block(0, x, 1, 1)) == -1                  # block 0 is a refresh block
     assert code(lambda: hero.hero_extrapolate_block(2, x, 1, 0)) == -1                  # d = 0
@@ -206,3 +208,77 @@ def test_many_contexts_do_not_leak_device_memory():
     torch.cuda.synchronize()
     torch.cuda.empty_cache()
     assert torch.cuda.mem_get_info()[0] >= free0 - (8 << 20)
+
+
+def test_partial_refresh_needs_a_full_pass_or_planted_caches():
+    """Eq. 3 merges fresh rows with the block's cache: until the block has had a full pass (or all four
+    caches were planted) a partial refresh is a call-order error, and hero_reset brings that state back."""
+    h = H()
+    cfgd = dict(S.CONFIGS["tiny"])
+    _, hero, _ = make_pair(cfgd)
+    cfg = O.Config.from_dict(cfgd)
+    x = to_dev(S.tokens(cfgd), "fp32")
+    t = to_dev(S.temb(cfgd, 0), "fp32")
+    idx = torch.arange(cfg.n_text, cfg.n_text + 8, dtype=torch.int32, device="cuda")
+
+    def code(fn):
+        with pytest.raises(h.HeroError) as e:
+            fn()
+        return e.value.code
+
+    assert code(lambda: hero.hero_refresh_block(0, x, t, idx)) == -4
+    zeros = torch.zeros(cfg.batch, cfg.n_rows, cfg.hidden)
+    for name in ("k", "v", "g_attn"):
+        hero.hero_state_set(0, name, zeros)
+    assert code(lambda: hero.hero_refresh_block(0, x, t, idx)) == -4                    # G_ffn still missing
+    hero.hero_state_set(0, "g_ffn", zeros)
+    hero.hero_refresh_block(0, x, t, idx)                                               # all four planted: fine
+    hero.hero_reset()
+    assert code(lambda: hero.hero_refresh_block(0, x, t, idx)) == -4
+    hero.hero_refresh_block(0, x, t)                                                    # full pass
+    hero.hero_refresh_block(0, x, t, idx)
+    hero.hero_refresh_block(0, x, t, idx, 0)
+    hero.hero_check_status()
+    hero.close()
+
+
+def test_a_wait_that_runs_out_is_reported_once_and_the_next_calls_are_healthy():
+    """The give-up path, made to happen harmlessly: one thread block waits 50 microseconds on a barrier
+    nobody completes, through the helper the tensor-core kernels use; it must raise the status word and
+    RETURN.  The host then reports HERO_ERR_TIMEOUT exactly once, and the kernels that share the word run
+    normally afterwards."""
+    h = H()
+    # the isolated calls' word
+    h.hero_isolated_status()
+    h.hero_selftest_wait_timeout(50)
+    with pytest.raises(h.HeroError) as e:
+        h.hero_isolated_status()
+    assert e.value.code == -6
+    h.hero_isolated_status()                                          # the word was cleared by the report
+    g = torch.Generator(device="cuda").manual_seed(3)
+    q, k, v = (torch.randn(1, n, 64, device="cuda", generator=g).bfloat16() for n in (70, 200, 200))
+    o = torch.full_like(q, float("nan"))
+    h.hero_attention_bf16(q, k, v, o, 1)
+    h.hero_isolated_status()
+    want = torch.softmax(q.float()[0] @ k.float()[0].T / 8.0, -1) @ v.float()[0]
+    assert float((o.float()[0] - want).norm() / want.norm()) <= 1e-2
+    # a context's word
+    cfgd = dict(n_blocks=1, n_shallow=1, hidden=128, n_heads=2, head_dim=64, ffn_dim=256, temb_dim=64, batch=1,
+                frames=1, grid_h=4, grid_w=4, n_text=2, patch_h=2, patch_w=2, ratio_num=1, ratio_den=4,
+                quota_mode=0, warmup_full_steps=2, full_interval=0, dtype="bf16", has_gate=0, seed=2, steps=3)
+    orc, hero, _ = make_pair(cfgd)
+    hero.hero_check_status()
+    hero.hero_selftest_wait_timeout(50)
+    with pytest.raises(h.HeroError) as e:
+        hero.hero_check_status()
+    assert e.value.code == -6
+    hero.hero_check_status()
+    x_host = S.tokens(cfgd)
+    for s in range(3):
+        temb = S.temb(cfgd, s)
+        want = orc.step(s, x_host, temb)
+        x = to_dev(x_host, "bf16")
+        hero.hero_step(s, x, to_dev(temb, "bf16"))
+        hero.hero_check_status()
+        assert rel_l2(to_host(x), want) <= 3e-2, s
+    hero.close()

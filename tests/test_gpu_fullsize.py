@@ -23,10 +23,15 @@ def H():
 
 
 CASES = {
+    "cogvideox_block_10": dict(S.CONFIGS["block"], ratio_num=1, ratio_den=10),
     "cogvideox_block_25": dict(S.CONFIGS["block"], ratio_num=1, ratio_den=4),
+    "cogvideox_block_50": dict(S.CONFIGS["block"], ratio_num=1, ratio_den=2),
     "cogvideox_block_25_qk_norm_rope": dict(S.CONFIGS["block"], ratio_num=1, ratio_den=4, qk_norm=1, rope=1),
     "cogvideox_block_25_attend_refreshed": dict(S.CONFIGS["block"], ratio_num=1, ratio_den=4, attend_mode=1),
     "aether_block_10": dict(S.CONFIGS["aether"], n_blocks=1, n_shallow=1, ratio_num=1, ratio_den=10, full_interval=0),
+    "aether_block_25": dict(S.CONFIGS["aether"], n_blocks=1, n_shallow=1, full_interval=0),
+    # the paper's own hyper-parameters: 2x3 patches, R = 0.2 rounded half up per patch (one token of six), 11 frames
+    "paper_hp_block": dict(S.CONFIGS["paper_hp"], n_blocks=1, n_shallow=1, full_interval=0),
 }
 
 
@@ -88,4 +93,100 @@ def test_refresh_block_full_size_sampled(name):
         assert np.array_equal(got[key][:, keep], val[:, keep].astype(np.float64)), key
     assert rel_l2(got_x[:, keep], want_x[:, keep]) <= 2 ** -8              # one bf16 rounding of the sum
     assert np.isfinite(got_x).all()
+    hero.close()
+
+
+def test_full_pass_full_size_sampled():
+    """Algorithm 1's "initial caching" pass at the one-block workload's full size (d_idx = NULL, all 17776
+    rows of both batch items: the launch the benchmark's full step times): K and V of EVERY row are compared,
+    the branch outputs and the residual stream on sampled rows (text rows, first and last row included)
+    that the oracle computes one by one."""
+    cfgd = dict(S.CONFIGS["block"])
+    cfg = O.Config.from_dict(cfgd)
+    B, N, D = cfg.batch, cfg.n_rows, cfg.hidden
+    weights = [S.block_weights(cfgd, 0)]
+    orc = O.HeroOracle(cfg, weights)
+    h = H()
+    hero = h.Hero(cfgd, [h.device_weights(weights[0], "bf16")])
+    rng = np.random.default_rng(23)
+    sample = np.unique(np.concatenate([rng.choice(N, 20, replace=False), [0, 1, cfg.n_text - 1, cfg.n_text, N - 1]]))
+    x_host = S.tokens(cfgd)
+    temb = S.temb(cfgd, 0)
+    x_dev = to_dev(x_host, "bf16")
+    hero.hero_refresh_block(0, x_dev, to_dev(temb, "bf16"))
+    hero.hero_check_status()
+    want_x = orc.block_refresh(0, x_host.astype(np.float64), temb, None, rows_out=sample)
+    st = orc.blocks[0]
+    for key, ref in (("k", st.k_cache), ("v", st.v_cache)):
+        got = to_host(hero.hero_state_get(0, key))
+        assert np.isfinite(got).all()
+        assert rel_l2(got, ref) <= BF16_TOL, key
+        for b in range(B):                                   # per batch item and on row bands, not only in total
+            for lo in range(0, N, 4096):
+                assert rel_l2(got[b, lo:lo + 4096], ref[b, lo:lo + 4096]) <= BF16_TOL, (key, b, lo)
+        del got
+    got_ga, got_gf = to_host(hero.hero_state_get(0, "g_attn")), to_host(hero.hero_state_get(0, "g_ffn"))
+    got_x = to_host(x_dev)
+    assert np.isfinite(got_ga).all() and np.isfinite(got_gf).all() and np.isfinite(got_x).all()
+    assert rel_l2(got_ga[:, sample], st.g[0][:, sample]) <= BF16_TOL
+    assert rel_l2(got_gf[:, sample], st.g[1][:, sample]) <= BF16_TOL
+    assert rel_l2(got_x[:, sample], want_x[:, sample]) <= BF16_TOL
+    for r in sample[:6]:
+        assert rel_l2(got_ga[:, r], st.g[0][:, r]) <= BF16_TOL, r
+        assert rel_l2(got_gf[:, r], st.g[1][:, r]) <= BF16_TOL, r
+    assert np.array_equal(hero.hero_state_get(0, "ages").numpy(), np.zeros(cfg.n_video, np.uint16))
+    hero.close()
+
+
+def test_grouped_deep_pass_full_size_sampled():
+    """Eq. 5 for a stack of 28 extrapolated blocks at [2, 17776, 3072] bf16: the one launch that carries all
+    deep blocks of the 42-block workload's cached step (56 history pairs streamed past x).  The histories are
+    what two full passes leave on the device; every history tensor is read back once and sampled, the oracle
+    applies Eq. 5 to the samples and adds them in block order.  Checked twice: through hero_step, and through
+    hero_step_host, which runs the pass over four row ranges and copies each back while the next is computed.
+    The real gap d = 3 and k = 2 are planted in the step record so that the slope is not the trivial one."""
+    n_deep = 28
+    cfgd = dict(S.CONFIGS["dit42"], n_blocks=n_deep, n_shallow=0, full_interval=0)
+    cfg = O.Config.from_dict(cfgd)
+    B, N, D = cfg.batch, cfg.n_rows, cfg.hidden
+    h = H()
+    w_host = S.block_weights(cfgd, 0)
+    w_dev = h.device_weights(w_host, "bf16")
+    hero = h.Hero(cfgd, [w_dev] * n_deep)          # every block borrows the same weights: only the histories matter here
+    x = to_dev(S.tokens(cfgd), "bf16")
+    for s in range(2):                              # two "initial caching" passes fill both history slots
+        hero.hero_step(s, x, to_dev(S.temb(cfgd, s), "bf16"))
+    hero.hero_check_status()
+    hero.hero_state_set(0, "steps", torch.tensor([2, 0, 3], dtype=torch.int32))   # full steps at 0 and 3
+    k, d = 2, 3
+    rng = np.random.default_rng(5)
+    n_el = B * N * D
+    # sampled flat elements: random ones, the first and last packets, and the seams of the four-piece route
+    per = ((n_el + 3) // 4 + 4095) // 4096 * 4096                             # length of one piece
+    seams = np.concatenate([[p * per - 1, p * per] for p in range(1, 4)])
+    flat = np.unique(np.concatenate([rng.choice(n_el, 4000, replace=False), np.arange(16), n_el - 1 - np.arange(16), seams]))
+    flat_t = torch.from_numpy(flat)
+    pick = lambda t: t.reshape(-1)[flat_t].double().numpy()                  # sampled elements as float64
+    x_before = x.clone()
+    want = pick(x_before.cpu())
+    largest = 0.0
+    for l in range(n_deep):
+        for br in ("g_attn", "g_ffn"):
+            last = pick(hero.hero_state_get(l, br))
+            prev = pick(hero.hero_state_get(l, br + "_prev"))
+            assert not np.array_equal(last, prev)
+            want = want + O.extrapolate(prev, last, k, d)
+            largest = max(largest, np.abs(want).max())
+    temb = to_dev(S.temb(cfgd, 5), "bf16")
+    x_a = x_before.clone()
+    hero.hero_step(5, x_a, temb)
+    hero.hero_check_status()
+    got = pick(x_a.cpu())
+    assert np.isfinite(got).all()
+    assert np.abs(got - want).max() <= 1e-2 * largest                       # one bf16 rounding of the sum
+    assert rel_l2(got, want) <= 5e-3
+    h_x = x_before.cpu().pin_memory()
+    hero.hero_step_host(5, h_x, temb.cpu().pin_memory())
+    hero.hero_check_status()
+    assert torch.equal(h_x, x_a.cpu())                                      # the four-piece route: same bits
     hero.close()

@@ -6,7 +6,7 @@ import torch
 
 from oracle import hero_oracle as O
 from workloads import synthetic as S
-from tests.util import rel_max, to_dev, to_host
+from tests.util import rel_l2, rel_max, to_dev, to_host
 
 pytestmark = pytest.mark.gpu
 
@@ -186,3 +186,35 @@ def test_select_bit_exact_on_random_geometries(case):
         assert (got[n:] == -1).all()
         assert np.array_equal(hero.hero_state_get(0, "ages").numpy(), ages), (cfgd, call)
     hero.close()
+
+
+# ---------------------------------------------------------------- gather + LayerNorm + modulate (Eq. 2's prologue)
+@pytest.mark.parametrize("dtype,B,N,D,n_sel,with_add", [
+    ("fp32", 1, 40, 128, 9, False), ("fp32", 2, 33, 260, 33, True),        # generic kernel (row through shared memory)
+    ("bf16", 2, 50, 256, 17, True), ("bf16", 1, 20, 1000, 20, False),      # generic kernel, bf16
+    ("bf16", 2, 300, 1024, 77, False), ("bf16", 2, 123, 2048, 50, True),   # one warp per row, 4 / 8 packets per lane
+    ("bf16", 2, 500, 3072, 259, True), ("bf16", 3, 64, 3072, 64, False),   # the CogVideoX width, ragged last CTA
+    ("bf16", 1, 40, 4096, 13, True)])
+def test_gather_ln_modulate_matches_oracle(dtype, B, N, D, n_sel, with_add):
+    rng = np.random.default_rng(N * 7 + D + n_sel)
+    rnd = (lambda a: S.round_bf16(a.astype(np.float32))) if dtype == "bf16" else (lambda a: a.astype(np.float32))
+    x = rnd(rng.standard_normal((B, N, D)) * 2.0 + 0.5)
+    add = rnd(rng.standard_normal((B, N, D)) * 0.3) if with_add else None
+    idx = np.sort(rng.choice(N, n_sel, replace=False)).astype(np.int32)
+    mod = rng.standard_normal((B, 4 * D)).astype(np.float32) * 0.5          # shift | scale | two unused chunks
+    cfg = O.Config(n_blocks=1, n_shallow=1, hidden=D, n_heads=1, head_dim=D, ffn_dim=8, temb_dim=8, batch=B,
+                   frames=1, grid_h=1, grid_w=1, n_text=0, patch_h=1, patch_w=1, ratio_num=1, ratio_den=1)
+    mod_d = torch.from_numpy(mod).cuda()
+    out = torch.full((B, n_sel, D), float("nan"), device="cuda", dtype=torch.bfloat16 if dtype == "bf16" else torch.float32)
+    H().hero_gather_ln_modulate(to_dev(x, dtype), None if add is None else to_dev(add, dtype),
+                                torch.from_numpy(idx).cuda(), mod_d[:, :D], mod_d[:, D:2 * D], out)
+    torch.cuda.synchronize()
+    got = to_host(out)
+    for b in range(B):
+        rows = x[b, idx].astype(np.float64) + (0.0 if add is None else add[b, idx].astype(np.float64))
+        want = O.layernorm_modulate(cfg, rows, mod[b, :D].astype(np.float64), mod[b, D:2 * D].astype(np.float64))
+        if dtype == "bf16":        # fp32 statistics, one bf16 rounding of the result
+            assert np.abs(got[b] - want).max() <= 2 ** -8 * np.abs(want).max() + 1e-6, b
+            assert rel_l2(got[b], want) <= 3e-3
+        else:
+            assert np.abs(got[b] - want).max() <= 2e-5 * np.abs(want).max(), b

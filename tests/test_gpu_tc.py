@@ -62,7 +62,8 @@ def test_gemm_many_tiles_per_cta():
                                            # second tile of the last group is empty, one row full, or full
                                            (1, 129, 300, 2), (2, 255, 193, 1), (1, 256, 97, 2), (1, 257, 300, 1),
                                            (2, 384, 200, 1), (1, 385, 290, 2), (1, 640, 100, 1)])
-def test_attention_matches_oracle(B, n_q, N, heads):
+@pytest.mark.parametrize("entry", ["hero_attention_bf16", "hero_attention_bf16_safe"])
+def test_attention_matches_oracle(B, n_q, N, heads, entry):
     rng = np.random.default_rng(B * 7 + n_q + N)
     D = heads * 64
     q = S.round_bf16(rng.standard_normal((B, n_q, D)).astype(np.float32))
@@ -71,7 +72,7 @@ def test_attention_matches_oracle(B, n_q, N, heads):
     cfg = O.Config(n_blocks=1, n_shallow=1, hidden=D, n_heads=heads, head_dim=64, ffn_dim=8, temb_dim=8, batch=B,
                    frames=1, grid_h=1, grid_w=1, n_text=0, patch_h=1, patch_w=1, ratio_num=1, ratio_den=1)
     o = torch.full((B, n_q, D), float("nan"), device="cuda", dtype=torch.bfloat16)
-    H().hero_attention_bf16(to_dev(q, "bf16"), to_dev(k, "bf16"), to_dev(v, "bf16"), o, heads)
+    getattr(H(), entry)(to_dev(q, "bf16"), to_dev(k, "bf16"), to_dev(v, "bf16"), o, heads)
     H().hero_isolated_status()
     got = to_host(o)
     assert np.isfinite(got).all()
@@ -95,15 +96,20 @@ def test_attention_peaked_rows():
 
 
 @pytest.mark.parametrize("N", [960, 1000, 97, 193])
-def test_attention_scores_that_keep_growing(N):
-    """Keys whose scores grow steadily along the sequence: the running maximum has to move again and again
-    (by more than the 2^8 slack), so the accumulator is rescaled in many key tiles, on both tile parities,
-    including the ragged last tile; rows with a flat score profile sit in the same warps."""
+@pytest.mark.parametrize("entry,top", [("hero_attention_bf16", 60.0), ("hero_attention_bf16_safe", 60.0),
+                                       ("hero_attention_bf16", 200.0)])
+def test_attention_scores_that_keep_growing(N, entry, top):
+    """Keys whose scores grow steadily along the sequence (by `top` in natural-log units from the first key to
+    the last).  In the safe kernel the running maximum has to move again and again (by more than the 2^8
+    slack), so the accumulator is rescaled in many key tiles, on both tile parities, including the ragged
+    last tile; rows with a flat score profile sit in the same warps.  The fast kernel keeps the first tile's
+    maximum: a rise of 60 stays inside its 2^100 range and is computed there, a rise of 200 is not, so the
+    climbing rows' thread blocks are handed to the safe kernel and the flat and descending ones are not."""
     rng = np.random.default_rng(N)
     n_q, D = 200, 64
     base = rng.standard_normal(D).astype(np.float32)
     base /= np.linalg.norm(base)
-    ramp = np.linspace(0.0, 60.0, N, dtype=np.float32)[:, None]                    # score ~ 8 * ramp * |q.base|
+    ramp = np.linspace(0.0, top, N, dtype=np.float32)[:, None]                     # score ~ 8 * ramp * |q.base|
     k = S.round_bf16((rng.standard_normal((1, N, D)) * 0.3 + ramp * base).astype(np.float32))
     v = S.round_bf16(rng.standard_normal((1, N, D)).astype(np.float32))
     q = rng.standard_normal((1, n_q, D)).astype(np.float32) * 0.3
@@ -113,13 +119,41 @@ def test_attention_scores_that_keep_growing(N):
     cfg = O.Config(n_blocks=1, n_shallow=1, hidden=D, n_heads=1, head_dim=64, ffn_dim=8, temb_dim=8, batch=1,
                    frames=1, grid_h=1, grid_w=1, n_text=0, patch_h=1, patch_w=1, ratio_num=1, ratio_den=1)
     o = torch.full((1, n_q, D), float("nan"), device="cuda", dtype=torch.bfloat16)
-    H().hero_attention_bf16(to_dev(q, "bf16"), to_dev(k, "bf16"), to_dev(v, "bf16"), o, 1)
+    getattr(H(), entry)(to_dev(q, "bf16"), to_dev(k, "bf16"), to_dev(v, "bf16"), o, 1)
     H().hero_isolated_status()
     got = to_host(o)[0]
     assert np.isfinite(got).all()
     want = O.attention(cfg, q[0].astype(np.float64), k[0].astype(np.float64), v[0].astype(np.float64))
     assert rel_l2(got, want) <= 1e-2
     assert np.abs(got - want).max() <= 3e-2 * np.abs(want).max()
+
+
+def test_attention_one_row_out_of_range_sends_only_its_thread_block_to_the_fallback():
+    """Three thread blocks of queries; one row of the middle one meets a key, late in the sequence, whose score
+    beats everything in the first key tile by far more than 2^100.  The result must be right everywhere: that
+    block through the fallback kernel, the other two straight from the fast one."""
+    rng = np.random.default_rng(77)
+    n_q, N, D = 700, 1500, 64
+    q = rng.standard_normal((1, n_q, D)).astype(np.float32)
+    k = rng.standard_normal((1, N, D)).astype(np.float32)
+    v = rng.standard_normal((1, N, D)).astype(np.float32)
+    k[0, 1234] = 16.0 * q[0, 300] / np.linalg.norm(q[0, 300])     # |k| = 16, along q
+    q[0, 300] *= 16.0 / np.linalg.norm(q[0, 300])                  # |q| = 16: q.k / 8 = 32 here, a few units elsewhere
+    q[0, 300] *= 8.0                                               # ... and 256 after this
+    q, k, v = S.round_bf16(q), S.round_bf16(k), S.round_bf16(v)
+    cfg = O.Config(n_blocks=1, n_shallow=1, hidden=D, n_heads=1, head_dim=64, ffn_dim=8, temb_dim=8, batch=1,
+                   frames=1, grid_h=1, grid_w=1, n_text=0, patch_h=1, patch_w=1, ratio_num=1, ratio_den=1)
+    s300 = (q[0, 300].astype(np.float64) @ k[0].astype(np.float64).T) / 8.0
+    assert s300[1234] - s300[:96].max() > 150.0                    # far beyond the fast kernel's range
+    o = torch.full((1, n_q, D), float("nan"), device="cuda", dtype=torch.bfloat16)
+    H().hero_attention_bf16(to_dev(q, "bf16"), to_dev(k, "bf16"), to_dev(v, "bf16"), o, 1)
+    H().hero_isolated_status()
+    got = to_host(o)[0]
+    assert np.isfinite(got).all()
+    want = O.attention(cfg, q[0].astype(np.float64), k[0].astype(np.float64), v[0].astype(np.float64))
+    for lo in (0, 256, 512):
+        assert rel_l2(got[lo:lo + 256], want[lo:lo + 256]) <= 1e-2, lo
+    assert np.abs(got[300] - v[0, 1234]).max() <= 2e-2             # that row returns the one key's value
 
 
 # ---------------------------------------------------------------- bf16 blocks

@@ -11,8 +11,11 @@ of allocated device memory unchanged.  It is named to be collected last.
 """
 import ctypes as C
 
+import numpy as np
 import pytest
 import torch
+
+from oracle import hero_oracle as O
 
 pytestmark = pytest.mark.gpu
 
@@ -51,6 +54,34 @@ def test_static_attention_matches_allocating_entry_point_twice():
         assert torch.equal(got, want), call
         err = (got.float() - want.float()).norm() / want.float().norm()
         assert float(err) <= 1e-2
+        # and against the definition itself (the CPU oracle's softmax(q k^T / 8) v per head), not only
+        # against the other entry point
+        cfg = O.Config(n_blocks=1, n_shallow=1, hidden=heads * 64, n_heads=heads, head_dim=64, ffn_dim=8, temb_dim=8,
+                       batch=B, frames=1, grid_h=1, grid_w=1, n_text=0, patch_h=1, patch_w=1, ratio_num=1, ratio_den=1)
+        for b in range(B):
+            ref = O.attention(cfg, *(t[b].float().cpu().numpy().astype(np.float64) for t in (q, k, v)))
+            out = got[b].float().cpu().numpy().astype(np.float64)
+            assert np.linalg.norm(out - ref) / np.linalg.norm(ref) <= 1e-2, (call, b)
+
+
+def test_static_attention_left_asynchronous_is_polled_without_allocating():
+    """A caller that must not block passes no give-up pointer; the verdict is fetched later with
+    hero_attention_bf16_static_status, which allocates nothing either."""
+    h = H()
+    B, n_q, N, heads = 1, 300, 700, 2                   # 2 query groups x 2 heads = 4 thread blocks
+    q, k, v = _inputs(B, n_q, N, heads, 55)
+    want = torch.empty_like(q)
+    h.hero_attention_bf16(q, k, v, want, heads)
+    h.hero_isolated_status()
+    got = torch.full_like(q, float("nan"))
+    h.hero_attention_bf16_static(q, k, v, got, heads)   # set-up done, nothing left to load
+    free_before = torch.cuda.mem_get_info()[0]
+    got.fill_(float("nan"))
+    h.hero_attention_bf16_static(q, k, v, got, heads, check=False)
+    gave_up, records = h.hero_attention_bf16_static_status(n_records=4)
+    assert torch.cuda.mem_get_info()[0] == free_before
+    assert gave_up == 0 and records == [0, 0, 0, 0]
+    assert torch.equal(got, want)
 
 
 def test_static_attention_refuses_what_its_scratch_cannot_serve():
