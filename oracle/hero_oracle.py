@@ -20,9 +20,22 @@ function (and collected in the design notes):
   * text rows are never refreshed on cached steps;
   * cached steps extrapolate with the real gap between the last two full steps.
 
-Parity pins: every function below is pinned by tests/test_oracle_*.py except the
-quality of the approximation on real videos (VBench, depth, pose), which needs the
-paper's weights and datasets: parity unpinned for that claim only.
+Parity pins: every function below is pinned by tests/test_oracle_*.py against something
+other than itself (values the paper prints, closed forms, invariants, library routines,
+brute force), with these exceptions, which are PARITY UNPINNED because the paper fixes
+nothing to pin them to:
+  * the quality of the approximation on real videos (VBench, depth, pose): needs the
+    paper's weights and datasets;
+  * rope_sections / rope_angles (opt-in, off in every listed workload): the paper does not
+    mention positional embeddings; the split of the rotary pairs over (frame, row, column)
+    and the frequency base are this build's statement of the base model's scheme, and the
+    tests only check them for internal consistency (fixed points, shift invariance, the
+    same formula typed a second time);
+  * token_hash's composition (seed ^ block, + call, + token through three mixer rounds): the
+    paper names no generator; the mixer itself is pinned (inverse, avalanche), the way it is
+    keyed only statistically;
+  * stability_scores' min-max normalisation: Sec. 4.1 states the range and the direction of
+    the score, not the formula.
 """
 from __future__ import annotations
 
@@ -468,9 +481,6 @@ class HeroOracle:
 
 
 # =============================================================================
-# The uncached step (Eq. 2 applied to every row, nothing stored)
-# =============================================================================
-# =============================================================================
 # Diagnostics (Sec. 4.1, hierarchical feature analysis; Fig. 4)
 # =============================================================================
 def second_difference_variance(features):
@@ -501,6 +511,9 @@ def extrapolation_error(g_prev, g_last, g_true, k: int, d: int):
     return float(np.sqrt((e ** 2).sum() / (np.asarray(g_true, F64) ** 2).sum()))
 
 
+# =============================================================================
+# The uncached step (Eq. 2 applied to every row, nothing stored)
+# =============================================================================
 def uncached_forward(cfg: Config, weights, x, temb):
     """Plain DiT block stack with no cache at all; written separately from
     HeroOracle so that "refresh ratio 1 with extrapolation off" can be checked

@@ -155,28 +155,41 @@ def test_call_order_and_argument_errors():
     hero.close()
 
 
-def test_paper_hyperparameters_small_model():
-    """The paper's own setting in miniature: 2x3 patches, R = 0.2 with round-half-up quotas (one token per
-    full patch), three of four blocks refreshed, a full step every M = 2 steps; 9 steps through hero_step."""
+@pytest.mark.parametrize("name,M,batch,steps,full_at", [
+    ("planning_M2", 2, 2, 9, [0, 1, 3, 5, 7]),          # visual planning: the guidance pair, M = 2
+    ("planning_M3", 3, 2, 11, [0, 1, 4, 7, 10]),        # M = 3: cached steps with k = 1 and k = 2, gap d = 3
+    ("reconstruction_M2", 2, 1, 9, [0, 1, 3, 5, 7]),    # reconstruction: one sequence, no guidance pair
+    ("reconstruction_M3", 3, 1, 11, [0, 1, 4, 7, 10])])
+def test_paper_hyperparameters_small_model(name, M, batch, steps, full_at):
+    """The paper's own settings (Sec. 5.1) in miniature: 2x3 patches, R = 0.2 with round-half-up quotas (one
+    token per full patch), three of four blocks refreshed, a full step every M = 2 or 3 steps, with and
+    without the guidance pair; through hero_step, every step against the oracle, with the schedule (which
+    steps are full, and the k and d the extrapolation therefore uses) checked against the expected list."""
     cfgd = dict(S.CONFIGS["tiny"], frames=2, grid_h=6, grid_w=9, patch_h=2, patch_w=3, ratio_num=1, ratio_den=5,
-                quota_mode=1, n_shallow=3, full_interval=2, steps=9, seed=77)
+                quota_mode=1, n_shallow=3, full_interval=M, batch=batch, steps=steps, seed=77)
     orc, hero, _ = make_pair(cfgd)
     cfg = O.Config.from_dict(cfgd)
     assert O.n_selected(cfg, 0) == cfg.n_video // 6
     x_host = S.tokens(cfgd)
-    n_full = 0
-    for s in range(cfgd["steps"]):                       # full at 0, 1, 3, 5, 7; cached at 2, 4, 6, 8
+    seen_full, seen_kd = [], set()
+    for s in range(cfgd["steps"]):
         temb = S.temb(cfgd, s)
         want = orc.step(s, x_host, temb)
         x = to_dev(x_host, "fp32")
         assert hero.hero_is_full_step(s) == orc.is_full_step(s)
-        n_full += orc.is_full_step(s)
+        if orc.is_full_step(s):
+            seen_full.append(s)
         hero.hero_step(s, x, to_dev(temb, "fp32"))
         assert rel_l2(to_host(x), want) <= FP32_TOL, s
+        n_full, s_prev, s_last = (int(v) for v in hero.hero_state_get(0, "steps"))
+        assert (n_full, s_last) == (len(seen_full), seen_full[-1])
+        if not orc.is_full_step(s):
+            seen_kd.add((s - s_last, s_last - s_prev))
         for l in range(cfgd["n_shallow"]):
             assert np.array_equal(hero.hero_state_get(l, "ages").numpy(), orc.blocks[l].ages)
             assert int(hero.hero_state_get(l, "calls")[0]) == orc.blocks[l].calls
-    assert n_full == 5
+    assert seen_full == full_at
+    assert seen_kd == ({(1, 1), (1, 2)} if M == 2 else {(1, 1), (2, 1), (1, 3), (2, 3)})
     hero.close()
 
 

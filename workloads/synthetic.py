@@ -45,13 +45,22 @@ CONFIGS = {
     # config 4: 42 blocks, 14 refresh at 25 % + 28 extrapolate, full step every 5
     "dit42": dict(_COGVIDEO, n_blocks=42, n_shallow=14, frames=13, ratio_num=1, ratio_den=4,
                   full_interval=5, seed=3, steps=50),
-    # config 5: Aether-shaped sequence, 17 latent frames, 48 latent channels
+    # config 5: Aether-shaped sequence, 17 latent frames (the 48 latent channels enter through the patch
+    # embedding, which is outside the block stack this library covers: the stack sees [B, N, hidden] tokens)
     "aether": dict(_COGVIDEO, n_blocks=42, n_shallow=14, frames=17, ratio_num=1, ratio_den=4,
-                   full_interval=5, seed=4, steps=50, latent_channels=48),
+                   full_interval=5, seed=4, steps=50),
     # the paper's own hyper-parameters (Sec. 5.1): 2x3 patches, R = 0.2 rounded per patch (Table 3 implies
     # round(6R) tokens), the first 20 blocks refreshed, a full step every M = 2 steps, 11 latent frames
     "paper_hp": dict(_COGVIDEO, n_blocks=42, n_shallow=20, frames=11, patch_h=2, patch_w=3, ratio_num=1,
                      ratio_den=5, quota_mode=1, full_interval=2, seed=5, steps=50),
+    # the same with the paper's other interval, M = 3 (visual planning: T = 50 steps, guidance pair)
+    "paper_hp_m3": dict(_COGVIDEO, n_blocks=42, n_shallow=20, frames=11, patch_h=2, patch_w=3, ratio_num=1,
+                        ratio_den=5, quota_mode=1, full_interval=3, seed=5, steps=50),
+    # reconstruction-shaped runs of the same model: one sequence (no guidance pair), T = 30 steps, M = 2 and 3
+    "paper_recon": dict(_COGVIDEO, n_blocks=42, n_shallow=20, frames=11, patch_h=2, patch_w=3, ratio_num=1,
+                        ratio_den=5, quota_mode=1, full_interval=2, seed=6, steps=30, batch=1),
+    "paper_recon_m3": dict(_COGVIDEO, n_blocks=42, n_shallow=20, frames=11, patch_h=2, patch_w=3, ratio_num=1,
+                           ratio_den=5, quota_mode=1, full_interval=3, seed=6, steps=30, batch=1),
 }
 
 
@@ -162,17 +171,6 @@ def cache_fill(cfg, tag: str, block: int, shape=None, std: float = 1.0) -> np.nd
     if shape is None:
         shape = (cfg["batch"], n_rows(cfg), cfg["hidden"])
     return normal(cfg["seed"], "cache_" + tag, shape, std=std, index=block, dtype=cfg["dtype"])
-
-
-def aether_latents(cfg) -> np.ndarray:
-    """Channel-concatenated latents [B, n_video, 4*C]: three modality groups
-    (colour, depth, raymap/action) with per-group scale 0.5 / 1.0 / 1.5 (config 5)."""
-    c = cfg.get("latent_channels", 48) * 4
-    z = normal(cfg["seed"], "latents", (cfg["batch"], n_video(cfg), c))
-    g = c // 3
-    z[..., :g] *= 0.5
-    z[..., 2 * g:] *= 1.5
-    return round_bf16(z) if cfg["dtype"] == "bf16" else z
 
 
 # ----------------------------------------------------------------------------
