@@ -22,20 +22,14 @@ function (and collected in the design notes):
 
 Parity pins: every function below is pinned by tests/test_oracle_*.py against something
 other than itself (values the paper prints, closed forms, invariants, library routines,
-brute force), with these exceptions, which are PARITY UNPINNED because the paper fixes
-nothing to pin them to:
-  * the quality of the approximation on real videos (VBench, depth, pose): needs the
-    paper's weights and datasets;
-  * rope_sections / rope_angles (opt-in, off in every listed workload): the paper does not
-    mention positional embeddings; the split of the rotary pairs over (frame, row, column)
-    and the frequency base are this build's statement of the base model's scheme, and the
-    tests only check them for internal consistency (fixed points, shift invariance, the
-    same formula typed a second time);
-  * token_hash's composition (seed ^ block, + call, + token through three mixer rounds): the
-    paper names no generator; the mixer itself is pinned (inverse, avalanche), the way it is
-    keyed only statistically;
-  * stability_scores' min-max normalisation: Sec. 4.1 states the range and the direction of
-    the score, not the formula.
+brute force).  Three of them implement a READING of a point on which the paper is silent,
+so their pins fix the function to the stated reading, not the reading to the paper:
+rope_sections / rope_angles (opt-in; first pair of an axis = the position in radians,
+linearity in the position, geometric frequencies spanning 1/10000, one section per axis),
+token_hash's keying (bijective in token, call and block, no interchangeable inputs, no
+serial correlation) and stability_scores' min-max normalisation (equally spaced variances
+give equally spaced scores).  PARITY UNPINNED: the quality of the approximation on real
+videos (VBench, depth, pose), which needs the paper's weights and datasets.
 """
 from __future__ import annotations
 

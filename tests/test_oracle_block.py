@@ -157,6 +157,38 @@ def test_rope_fixed_points_known_angles_and_shift_invariance():
     assert abs(dot(row(1, 2, 3), row(0, 1, 6)) - base) > 1e-3
 
 
+def test_rope_angles_closed_forms():
+    """What fixes the rotary angles without typing their formula again: every axis' first pair turns by
+    exactly `position` radians; angles are linear in the position; inside an axis the frequencies form a
+    geometric sequence whose ratio, taken to the power of the axis' pair count, is 1 / 10000; an axis' pairs
+    move with that axis' coordinate and no other; text rows have no angle.  A wrong split, base, index or
+    axis order fails one of these."""
+    cfg = small_cfg(rope=1, head_dim=64, n_heads=1, hidden=64, frames=5, grid_h=7, grid_w=9, n_text=4)
+    p_t, p_h, p_w = O.rope_sections(cfg)
+    assert (p_t, p_h, p_w) == (8, 12, 12) and p_t + p_h + p_w == cfg.head_dim // 2
+    row = lambda f, y, x: cfg.n_text + (f * cfg.grid_h + y) * cfg.grid_w + x
+    ang = lambda f, y, x: O.rope_angles(cfg, [row(f, y, x)])[0]
+    first = {0: 0, 1: p_t, 2: p_t + p_h}                        # first pair of each axis' section
+    a = ang(3, 5, 7)
+    assert a[first[0]] == 3.0 and a[first[1]] == 5.0 and a[first[2]] == 7.0
+    np.testing.assert_allclose(ang(4, 6, 8), 2.0 * ang(2, 3, 4), rtol=1e-14)              # linear in the position
+    np.testing.assert_allclose(ang(1, 2, 3) + ang(3, 4, 5), ang(4, 6, 8), rtol=1e-14)
+    one = ang(1, 1, 1)                                           # the frequencies themselves
+    for start, n in ((0, p_t), (p_t, p_h), (p_t + p_h, p_w)):
+        freq = one[start:start + n]
+        ratio = freq[1:] / freq[:-1]
+        np.testing.assert_allclose(ratio, ratio[0], rtol=1e-13)                           # geometric
+        assert 0.0 < ratio[0] < 1.0                                                       # falling with the pair index
+        np.testing.assert_allclose(ratio[0] ** n, 1.0e-4, rtol=1e-12)                     # n steps span the base
+    base = ang(2, 3, 4)
+    moved = [ang(3, 3, 4) != base, ang(2, 4, 4) != base, ang(2, 3, 5) != base]
+    sections = [slice(0, p_t), slice(p_t, p_t + p_h), slice(p_t + p_h, None)]
+    for axis in range(3):                                        # an axis' coordinate moves its own section only
+        for sec in range(3):
+            assert moved[axis][sections[sec]].all() == (axis == sec) and moved[axis][sections[sec]].any() == (axis == sec)
+    assert not O.rope_angles(cfg, np.arange(cfg.n_text)).any()   # text rows
+
+
 @pytest.mark.parametrize("extras", [dict(), dict(qk_norm=1, rope=1)])
 def test_ratio_one_without_extrapolation_equals_uncached_step(extras):
     """R = 1 makes S(z) = z; with text rows included and every block shallow, a cached
@@ -460,6 +492,15 @@ def test_stability_scores_order_range_and_invariances():
     np.testing.assert_allclose(O.stability_scores([f + 3.0 * t + 1.0 for f in layers]), sc, atol=1e-12)
     np.testing.assert_allclose(O.stability_scores([7.0 * f for f in layers]), sc, atol=1e-12)
     assert np.array_equal(O.stability_scores([layers[0], layers[0]]), np.ones(2))
+    # closed form of the normalisation: white noise of standard deviation s has second-difference variance
+    # 6 s^2, so layers with s^2 in arithmetic progression land on equally spaced scores 1, 1/2, 0 (up to
+    # sampling noise), and one more layer between two others moves none of theirs
+    big = rng.standard_normal((3, 300, 4000))
+    sc3 = O.stability_scores([big[0] * np.sqrt(1.0), big[1] * np.sqrt(2.0), big[2] * np.sqrt(3.0)])
+    np.testing.assert_allclose(sc3, [1.0, 0.5, 0.0], atol=2e-2)
+    sc4 = O.stability_scores([big[0], big[1] * np.sqrt(2.0), big[2] * np.sqrt(3.0), big[1] * np.sqrt(1.5)])
+    np.testing.assert_allclose(sc4[:3], sc3, atol=1e-12)
+    np.testing.assert_allclose(sc4[3], 0.75, atol=2e-2)
 
 
 def test_extrapolation_error_is_zero_on_linear_features_and_known_on_a_quadratic():

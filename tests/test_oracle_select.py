@@ -293,3 +293,32 @@ def test_oldest_first_prefers_age_over_any_draw_and_uses_the_draw_among_equals()
         rows, _ = O.select_tokens(O.Config.from_dict(dict(cfgd, seed=seed)), np.zeros(4, np.uint16), 0, 0)
         winners.add(int(rows[0]))
     assert winners == {0, 1, 2, 3}
+
+
+def test_every_input_of_the_draw_enters_it_and_none_collides():
+    """How the draw is keyed, without typing the composition again: for fixed other inputs the draw is a
+    bijection of the token index, of the call counter and of the block index (each passes through an invertible
+    mixer round after it is added), so no two tokens, calls or blocks share a draw; only the low 32 bits of the
+    seed matter; and the four inputs are not interchangeable (the draw of (block, call, token) = (a, b, c) is
+    not that of any permutation), which a transposed argument would break."""
+    seed = 0x1234ABCD
+    n = 1 << 12
+    assert len({O.token_hash(seed, 3, 5, v) for v in range(n)}) == n
+    assert len({O.token_hash(seed, 3, c, 77) for c in range(n)}) == n
+    assert len({O.token_hash(seed, b, 5, 77) for b in range(n)}) == n
+    assert O.token_hash(seed + (7 << 32), 3, 5, 77) == O.token_hash(seed, 3, 5, 77)
+    assert O.token_hash(seed ^ 1, 3, 5, 77) != O.token_hash(seed, 3, 5, 77)
+    import itertools
+    a, b, c = 2, 11, 301
+    draws = {perm: O.token_hash(seed, *perm) for perm in itertools.permutations((a, b, c))}
+    assert len(set(draws.values())) == 6
+    # consecutive tokens, calls and blocks give unrelated draws: the low bit of the draw is balanced and shows
+    # no correlation along any of the three axes (a dropped mixer round would leave a counter's pattern in it)
+    import numpy as np
+    for axis in range(3):
+        args = [[3, 5, 77] for _ in range(4096)]
+        for i, arg in enumerate(args):
+            arg[axis] = i
+        bits = np.array([O.token_hash(seed, *arg) & 1 for arg in args], dtype=np.float64)
+        assert abs(bits.mean() - 0.5) < 0.04
+        assert abs(np.corrcoef(bits[:-1], bits[1:])[0, 1]) < 0.06
