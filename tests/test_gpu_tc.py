@@ -61,7 +61,10 @@ def test_gemm_many_tiles_per_cta():
                                            # query counts around the 128-row tile and 256-row group edges: the
                                            # second tile of the last group is empty, one row full, or full
                                            (1, 129, 300, 2), (2, 255, 193, 1), (1, 256, 97, 2), (1, 257, 300, 1),
-                                           (2, 384, 200, 1), (1, 385, 290, 2), (1, 640, 100, 1)])
+                                           (2, 384, 200, 1), (1, 385, 290, 2), (1, 640, 100, 1),
+                                           # key counts around the 96-key tile and the 48-column split of a row between
+                                           # two threads: one half empty, one key in it, exactly one tile, one key more
+                                           (1, 100, 48, 1), (2, 70, 49, 2), (1, 100, 96, 1), (3, 129, 95, 1), (1, 33, 145, 1)])
 @pytest.mark.parametrize("entry", ["hero_attention_bf16", "hero_attention_bf16_safe"])
 def test_attention_matches_oracle(B, n_q, N, heads, entry):
     rng = np.random.default_rng(B * 7 + n_q + N)
