@@ -170,6 +170,7 @@ def test_grouped_deep_pass_full_size_sampled():
     x_before = x.clone()
     want = pick(x_before.cpu())
     largest = 0.0
+    sum_last, sum_prev = np.zeros(len(flat)), np.zeros(len(flat))             # for the collapsed stack below
     for l in range(n_deep):
         for br in ("g_attn", "g_ffn"):
             last = pick(hero.hero_state_get(l, br))
@@ -177,6 +178,8 @@ def test_grouped_deep_pass_full_size_sampled():
             assert not np.array_equal(last, prev)
             want = want + O.extrapolate(prev, last, k, d)
             largest = max(largest, np.abs(want).max())
+            sum_last += last
+            sum_prev += prev
     temb = to_dev(S.temb(cfgd, 5), "bf16")
     x_a = x_before.clone()
     hero.hero_step(5, x_a, temb)
@@ -189,4 +192,28 @@ def test_grouped_deep_pass_full_size_sampled():
     hero.hero_step_host(5, h_x, temb.cpu().pin_memory())
     hero.hero_check_status()
     assert torch.equal(h_x, x_a.cpu())                                      # the four-piece route: same bits
+    hero.close()
+
+    # The collapsed deep stack (deep_collapse = 1) at the same size and on the same inputs: its two fp32 sums must
+    # be the sums of the per-block branch outputs read above (Eq. 5 is linear, Sec. 4.4), and its one-pass
+    # cached step must land on the same values as the block-by-block oracle.
+    del hero
+    torch.cuda.empty_cache()
+    hero = h.Hero(dict(cfgd, deep_collapse=1), [w_dev] * n_deep)
+    x = to_dev(S.tokens(cfgd), "bf16")
+    for s in range(2):
+        hero.hero_step(s, x, to_dev(S.temb(cfgd, s), "bf16"))
+    hero.hero_check_status()
+    assert torch.equal(x, x_before)                                          # same full steps, same bits
+    got_last, got_prev = pick(hero.hero_state_get(0, "stack_last")), pick(hero.hero_state_get(0, "stack_prev"))
+    scale = max(np.abs(sum_last).max(), 1e-30)
+    assert np.abs(got_last - sum_last).max() <= 2e-6 * scale                 # fp32 running sums of bf16 values
+    assert np.abs(got_prev - sum_prev).max() <= 2e-6 * scale
+    hero.hero_state_set(0, "steps", torch.tensor([2, 0, 3], dtype=torch.int32))
+    x_c = x_before.clone()
+    hero.hero_step(5, x_c, temb)
+    hero.hero_check_status()
+    got_c = pick(x_c.cpu())
+    assert np.abs(got_c - want).max() <= 1e-2 * largest
+    assert rel_l2(got_c, want) <= 5e-3
     hero.close()
