@@ -248,6 +248,16 @@ int hero_attention_bf16(const void *d_q, const void *d_k, const void *d_v, void 
 int hero_attention_bf16_safe(const void *d_q, const void *d_k, const void *d_v, void *d_o,
                              int B, int n_q, int N, int heads, void *stream);
 
+/* hero_attention_bf16 for a caller that has folded the softmax scale into its queries: d_q holds
+ * Q * log2(e) / sqrt(head_dim) (= Q * 0.18033688 at head_dim 64), so a score is the base-2 exponent of its
+ * weight and O = sum_j 2^(Q'.K_j) V_j / sum_j 2^(Q'.K_j), the same softmax (Sec. 4.3).  This is the form
+ * hero_step and hero_refresh_block use (their QKV projection writes q that way): the fast kernel then takes
+ * 2^score as it stands, with no row maximum at all.  Exact while every row's largest score lies within
+ * about +-100 (bf16 and fp32 share the exponent range); a row sum outside [2^-100, 2^100) hands its thread
+ * block to the second kernel, as above.  Shapes, layouts and errors as hero_attention_bf16. */
+int hero_attention_bf16_q_scaled(const void *d_q, const void *d_k, const void *d_v, void *d_o,
+                                 int B, int n_q, int N, int heads, void *stream);
+
 /* hero_attention_bf16 without any allocation (the paper has no counterpart: this entry point
  * exists for the sake of callers, not of the method).  hero_attention_bf16 obtains its status
  * word with cudaMalloc on first use; a caller that must never enter the CUDA allocator - a

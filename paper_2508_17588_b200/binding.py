@@ -25,7 +25,7 @@ EXPORTS = [
     "hero_init", "hero_reset", "hero_destroy", "hero_strerror", "hero_check_status", "hero_last_cuda_error",
     "hero_device_bytes", "hero_launch_count", "hero_profile_begin", "hero_profile_end", "hero_select_tokens", "hero_next_n_sel", "hero_refresh_block",
     "hero_extrapolate_block", "hero_extrapolate_deep_stack", "hero_step", "hero_step_host", "hero_is_full_step", "hero_extrapolate",
-    "hero_gather_rows", "hero_scatter_rows", "hero_gemm_bf16", "hero_attention_bf16", "hero_attention_bf16_safe", "hero_attention_bf16_static", "hero_attention_bf16_static_status",
+    "hero_gather_rows", "hero_scatter_rows", "hero_gemm_bf16", "hero_attention_bf16", "hero_attention_bf16_safe", "hero_attention_bf16_q_scaled", "hero_attention_bf16_static", "hero_attention_bf16_static_status",
     "hero_isolated_status", "hero_selftest_wait_timeout", "hero_gather_ln_modulate",
     "hero_state_get", "hero_state_set", "hero_second_difference_moments", "hero_extrapolation_error",
 ]
@@ -93,6 +93,7 @@ def load() -> C.CDLL:
         "hero_gemm_bf16": (i, [vp, vp, vp, vp, i, i, i, i, vp]),
         "hero_attention_bf16": (i, [vp, vp, vp, vp, i, i, i, i, vp]),
         "hero_attention_bf16_safe": (i, [vp, vp, vp, vp, i, i, i, i, vp]),
+        "hero_attention_bf16_q_scaled": (i, [vp, vp, vp, vp, i, i, i, i, vp]),
         "hero_attention_bf16_static": (i, [vp, vp, vp, vp, i, i, i, i, vp, ip]),
         "hero_attention_bf16_static_status": (i, [vp, ip, ip, i]),
         "hero_isolated_status": (i, [vp]),
@@ -336,6 +337,16 @@ def hero_attention_bf16_safe(q, k, v, o, heads: int):
     N = k.shape[1]
     _check(load().hero_attention_bf16_safe(_ptr(q), _ptr(k), _ptr(v), _ptr(o), B, n_q, N, heads, _stream()),
            "hero_attention_bf16_safe")
+    return o
+
+
+def hero_attention_bf16_q_scaled(q, k, v, o, heads: int):
+    """hero_attention_bf16 for queries that already carry the factor log2(e) / sqrt(head_dim)."""
+    _require_cuda()
+    B, n_q, _ = q.shape
+    N = k.shape[1]
+    _check(load().hero_attention_bf16_q_scaled(_ptr(q), _ptr(k), _ptr(v), _ptr(o), B, n_q, N, heads, _stream()),
+           "hero_attention_bf16_q_scaled")
     return o
 
 

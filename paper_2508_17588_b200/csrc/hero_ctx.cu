@@ -171,7 +171,7 @@ int run_attention(hero_ctx* c, const void* q, const void* k, const void* v, void
   const hero_config& g = c->cfg;
   LaunchScope scope(c, HERO_PROF_ATTENTION);
   if (g.dtype == HERO_DTYPE_BF16)
-    return launch_tc_attention(q, k, v, o, g.batch, n_q, c->N, g.n_heads, c->d_status, c->status_ctas, c->stream);
+    return launch_tc_attention(q, k, v, o, g.batch, n_q, c->N, g.n_heads, true, c->d_status, c->status_ctas, c->stream);
   return launch_simt_attention(q, k, v, o, g.batch, n_q, c->N, g.n_heads, g.head_dim, g.dtype, c->stream);
 }
 
@@ -241,9 +241,15 @@ int refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, const i
   o_qkv.ptr[1] = kdst;    o_qkv.ld[1] = D; o_qkv.scatter[1] = 1;
   o_qkv.ptr[2] = vdst;    o_qkv.ld[2] = D; o_qkv.scatter[2] = 1;
   o_qkv.seg_cols = D; o_qkv.idx = d_idx; o_qkv.n_sel = n_sel; o_qkv.n_rows = N;
+  // The tensor-core attention takes q with the softmax scale folded in (a score is then the exponent of its
+  // weight): by the projection's epilogue, or by the q/k treatment below when that runs and has the last word on q.
+  const bool fold_scale = g.dtype == HERO_DTYPE_BF16;
+  const bool qk_treated = g.qk_norm || g.rope;
+  if (fold_scale && !qk_treated) o_qkv.seg0_scale = kScoreScaleLog2;
   HERO_TRY(run_gemm(c, c->ws_a, w.w_qkv, w.b_qkv, M, 3 * D, D, o_qkv));
-  if (g.qk_norm || g.rope) {
+  if (qk_treated) {
     QkPrepArgs qa = {};
+    if (fold_scale) qa.q_scale = kScoreScaleLog2;
     qa.q = c->ws_q; qa.k = kdst; qa.idx = d_idx;
     if (g.qk_norm) { qa.qn_w = w.qn_w; qa.qn_b = w.qn_b; qa.kn_w = w.kn_w; qa.kn_b = w.kn_b; }
     qa.rope = g.rope ? c->rope_tab : nullptr;
@@ -263,8 +269,8 @@ int refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, const i
                 launch_gather_rows(vdst, c->att_list, c->kv_cmp[1], B, N, n_att, D, g.dtype, c->stream));
     LaunchScope scope(c, HERO_PROF_ATTENTION);
     if (g.dtype == HERO_DTYPE_BF16)
-      HERO_TRY(launch_tc_attention(c->ws_q, c->kv_cmp[0], c->kv_cmp[1], c->ws_o, B, n_sel, n_att, g.n_heads, c->d_status,
-                                   c->status_ctas, c->stream));
+      HERO_TRY(launch_tc_attention(c->ws_q, c->kv_cmp[0], c->kv_cmp[1], c->ws_o, B, n_sel, n_att, g.n_heads, true,
+                                   c->d_status, c->status_ctas, c->stream));
     else
       HERO_TRY(launch_simt_attention(c->ws_q, c->kv_cmp[0], c->kv_cmp[1], c->ws_o, B, n_sel, n_att, g.n_heads, g.head_dim,
                                      g.dtype, c->stream));
@@ -866,7 +872,17 @@ int hero_attention_bf16(const void* q, const void* k, const void* v, void* o, in
   if (!q || !k || !v || !o) return HERO_ERR_ARG;
   int* st = isolated_status();
   if (!st) return HERO_ERR_NOMEM;
-  return launch_tc_attention(q, k, v, o, B, n_q, N, heads, st, kIsolatedStatusCtas, (cudaStream_t)stream);
+  return launch_tc_attention(q, k, v, o, B, n_q, N, heads, false, st, kIsolatedStatusCtas, (cudaStream_t)stream);
+}
+
+int hero_attention_bf16_q_scaled(const void* q, const void* k, const void* v, void* o, int B, int n_q, int N,
+                                 int heads, void* stream) {
+  if (B < 0 || n_q < 0 || N <= 0 || heads <= 0) return HERO_ERR_ARG;
+  if (B == 0 || n_q == 0) return HERO_OK;
+  if (!q || !k || !v || !o) return HERO_ERR_ARG;
+  int* st = isolated_status();
+  if (!st) return HERO_ERR_NOMEM;
+  return launch_tc_attention(q, k, v, o, B, n_q, N, heads, true, st, kIsolatedStatusCtas, (cudaStream_t)stream);
 }
 
 int hero_attention_bf16_safe(const void* q, const void* k, const void* v, void* o, int B, int n_q, int N, int heads,
@@ -876,7 +892,7 @@ int hero_attention_bf16_safe(const void* q, const void* k, const void* v, void* 
   if (!q || !k || !v || !o) return HERO_ERR_ARG;
   int* st = isolated_status();
   if (!st) return HERO_ERR_NOMEM;
-  return launch_tc_attention_safe(q, k, v, o, B, n_q, N, heads, st, (cudaStream_t)stream);
+  return launch_tc_attention_safe(q, k, v, o, B, n_q, N, heads, false, st, (cudaStream_t)stream);
 }
 
 // Synchronise `stream` and report whether an isolated tensor-core call gave up on a wait.

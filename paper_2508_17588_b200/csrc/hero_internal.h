@@ -75,6 +75,7 @@ struct GemmOut {
   const float* gate;   // optional multiplier [B, gate_ld], indexed by column within the segment
   int gate_ld;
   int act;             // 0 = identity, 1 = GELU-tanh
+  float seg0_scale;    // when not 0: factor on the columns of segment 0 (applied after the bias, before rounding)
 };
 
 // Geometry of the selection problem (Sec. 4.3).
@@ -131,6 +132,7 @@ struct QkPrepArgs {
   int n_text, frames, grid_h, grid_w;
   int p_t, p_h, p_w;       // rotary pairs per axis
   float eps;
+  float q_scale;           // when not 0: factor on the finished q rows (the softmax scale, folded in here)
 };
 int launch_qk_prep(const QkPrepArgs& a, int dtype, cudaStream_t s);
 // list[i] = i for i < n_text, list[n_text + i] = idx[i] for i < n_sel (rows a literal Eq. 3 attends to)
@@ -167,10 +169,13 @@ int tc_init_driver_api();   // resolves cuTensorMapEncodeTiled once
 int launch_tc_gemm(const void* a, const void* w, const void* bias, int M, int Nout, int K,
                    const GemmOut& out, int* d_status, cudaStream_t s);
 // d_status: word 0 (give-up counter) followed by status_ctas per-CTA words
+// The tensor-core attention serves head_dim 64: a score s enters the softmax as 2^(s * kScoreScaleLog2).
+constexpr float kScoreScaleLog2 = 0.125f * 1.4426950408889634f;   // 1/sqrt(64) * log2(e)
+// q_prescaled: Q holds q * kScoreScaleLog2 (the softmax scale folded into the projection)
 int launch_tc_attention(const void* q, const void* k, const void* v, void* o, int B, int n_q, int N,
-                        int heads, int* d_status, int status_ctas, cudaStream_t s);
+                        int heads, bool q_prescaled, int* d_status, int status_ctas, cudaStream_t s);
 int launch_tc_attention_safe(const void* q, const void* k, const void* v, void* o, int B, int n_q, int N,
-                             int heads, int* d_status, cudaStream_t s);
+                             int heads, bool q_prescaled, int* d_status, cudaStream_t s);
 long long tc_attention_grid(int B, int n_q, int heads);   // CTAs of one attention launch
 
 // one thread block, no TMA, no TMEM: a bounded wait on a barrier nobody arms; raises *d_status and returns

@@ -103,10 +103,11 @@ __global__ void __launch_bounds__(256) qk_prep_kernel(QkPrepArgs a) {
         }
       }
     }
+    const float out_scale = (!which && a.q_scale != 0.f) ? a.q_scale : 1.0f;
 #pragma unroll
     for (int j = 0; j < kMaxPairsPerLane; ++j) {
       const int pr = lane + 32 * j;
-      if (pr < pairs) store_pair<T>(p + 2 * pr, v[j]);
+      if (pr < pairs) store_pair<T>(p + 2 * pr, make_float2(v[j].x * out_scale, v[j].y * out_scale));
     }
   }
 }
@@ -182,10 +183,11 @@ __global__ void __launch_bounds__(256) qk_prep_hd64_kernel(QkPrepArgs a, int n_c
         v[j].y = x * cs.y + y * cs.x;
       }
     }
+    const float out_scale = (!which[u] && a.q_scale != 0.f) ? a.q_scale : 1.0f;
     uint4 out;
     __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&out);
 #pragma unroll
-    for (int j = 0; j < 4; ++j) o2[j] = __float22bfloat162_rn(v[j]);
+    for (int j = 0; j < 4; ++j) o2[j] = __float22bfloat162_rn(make_float2(v[j].x * out_scale, v[j].y * out_scale));
     if (live[u]) *reinterpret_cast<uint4*>(ptr[u]) = out;
   }
 }

@@ -26,6 +26,10 @@
 //    (69 in natural-log units; bf16 and fp32 share their exponent range, so a large p loses no
 //    precision, and the final division by the row sum makes the result independent of the maximum
 //    used).  The row sum tells whether that held; a CTA in which it did not says so in its status word.
+//    In the step the QKV projection hands over q already multiplied by log2(e) / sqrt(64), so a score is
+//    the exponent of its weight: that instantiation (PRESCALED) takes p = 2^s as it stands - no maximum,
+//    no first-tile exchange, no multiply-add per pair of scores - and is exact while a row's largest score
+//    stays within about +-100; its row sum must then lie in [2^-100, 2^100), else the CTA is marked.
 //  * tc_attention_safe_kernel recomputes exactly those CTAs (same grid, every other CTA returns at
 //    once) with a running maximum that moves whenever a tile exceeds it by 2^8, rescaling the
 //    accumulator in TMEM; it is also the whole computation when no per-CTA status words are available.
@@ -174,7 +178,7 @@ __device__ __forceinline__ void fused_tile(uint32_t t_buf, float c, float neg_mc
 __global__ void __launch_bounds__(kAttThreads, 1)
 tc_attention_safe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                          const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ O, int n_q, int N,
-                         int heads, int* __restrict__ status, int* __restrict__ cta_words) {
+                         int heads, const float c, int* __restrict__ status, int* __restrict__ cta_words) {
   if (cta_words != nullptr && cta_words[blockIdx.x] != 1) return;      // block-uniform
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -280,7 +284,6 @@ tc_attention_safe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     const int t = (warp - kFirstSoftmaxWarp) >> 2;     // query tile of this softmax group
     const int quad = warp & 3;                         // TMEM lane quadrant this warp may touch
     const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)t * kTileCols;
-    const float c = 0.125f * 1.4426950408889634f;      // 1/sqrt(64) * log2(e)
     float m_used = -INFINITY, l_run = 0.f;
     bool ok = true;
     for (int j = 0; j < n_kv; ++j) {
@@ -381,6 +384,7 @@ constexpr int kHalf = kKT / 2;                   // score columns of a key tile 
 constexpr int kXchgFloats = kQTiles * kQT * 2;   // one slot per (query row, column half)
 constexpr size_t kFastSmem = kAttSmem + 2 * kXchgFloats * sizeof(float) + 64;
 constexpr float kRowSumLimit = 1.2676506e30f;    // 2^100: a row sum at or beyond it voids the fixed-maximum assumption
+constexpr float kRowSumFloor = 7.8886091e-31f;   // 2^-100: below it a row without a maximum has lost its small terms
 static_assert(kHalf % 16 == 0 && (kHalf / 16) % 2 == 1, "three 16-column reads per half: the ping-pong below ends on ra");
 
 // 2^x for two scores on the FMA pipe instead of the special-function unit (Cody-Waite reduction + a cubic).
@@ -396,7 +400,10 @@ static_assert(kHalf % 16 == 0 && (kHalf / 16) % 2 == 1, "three 16-column reads p
 #ifndef HERO_ATT_POLY_PAIRS
 #define HERO_ATT_POLY_PAIRS 1          // of every 8 pairs of scores (1 measured best: 2.22 ms against 2.40 with none, 2.33 with 2)
 #endif
-constexpr int kPolyPairs = HERO_ATT_POLY_PAIRS;
+#ifndef HERO_ATT_POLY_PAIRS_PRESCALED
+#define HERO_ATT_POLY_PAIRS_PRESCALED 2   // with the scale folded into q a pair costs the pipes one instruction less: 2 is best
+#endif
+constexpr int kPolyPairs = HERO_ATT_POLY_PAIRS, kPolyPairsPrescaled = HERO_ATT_POLY_PAIRS_PRESCALED;
 constexpr float kPolySpan = 250.0f, kPolyMagic = 12582912.0f - 125.0f;
 __device__ __forceinline__ float fma_sat(float a, float b, float c) {
   float y;
@@ -419,7 +426,8 @@ __device__ __forceinline__ float2 exp2_poly_pair(float s0, float s1, float cs, f
 // ahead), turned into p = 2^(s c - m c), summed, packed to bf16 and written back over the columns just read -
 // half h keeps its P in the first 24 columns of its own 48, so neither half ever writes what the other reads.
 // MASKED (the ragged last tile): columns at or beyond `valid` are keys that do not exist.
-template <bool MASKED>
+// PRESCALED: the scores are exponents already (x = s, see the kernel below), one instruction less per pair.
+template <bool MASKED, bool PRESCALED>
 __device__ __forceinline__ float half_tile(uint32_t t_s, int valid, const float2 c2, const float2 nm2, float cs, float bs) {
   float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
   uint32_t ra[16], rb[16];
@@ -434,10 +442,11 @@ __device__ __forceinline__ float half_tile(uint32_t t_s, int valid, const float2
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       float2 p;
-      if ((i * kPolyPairs) % 8 < kPolyPairs) {          // spread evenly over the chunk (resolved at compile time)
+      constexpr int kPoly = PRESCALED ? kPolyPairsPrescaled : kPolyPairs;
+      if ((i * kPoly) % 8 < kPoly) {                    // spread evenly over the chunk (resolved at compile time)
         p = exp2_poly_pair(__uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1]), cs, bs);
       } else {
-        const float2 x = __ffma2_rn(f2(cur[2 * i], cur[2 * i + 1]), c2, nm2);
+        const float2 x = PRESCALED ? f2(cur[2 * i], cur[2 * i + 1]) : __ffma2_rn(f2(cur[2 * i], cur[2 * i + 1]), c2, nm2);
         p = make_float2(ex2(x.x), ex2(x.y));
       }
       if (MASKED) {
@@ -454,6 +463,7 @@ __device__ __forceinline__ float half_tile(uint32_t t_s, int valid, const float2
   return (a01.x + a01.y) + (a23.x + a23.y);
 }
 
+template <bool PRESCALED>
 __global__ void __launch_bounds__(kFastThreads, 1)
 tc_attention_fast_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                          const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ O, int n_q, int N,
@@ -580,12 +590,13 @@ tc_attention_fast_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     const int row = quad * 32 + lane;                  // query row within the tile
     const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)t * kTileCols;
     uint64_t* my_pair = &pair_bar[t * 4 + quad];
-    const float c = 0.125f * 1.4426950408889634f;      // 1/sqrt(64) * log2(e)
+    const float c = PRESCALED ? 1.0f : kScoreScaleLog2;
     const float2 c2 = make_float2(c, c);
     float2 nm2 = make_float2(0.f, 0.f);
     const float cs = c / kPolySpan;
     float bs = 0.5f;
     float l_half = 0.f;
+    uint32_t pair_phase = 0;
     bool ok = true;
     for (int j = 0; j < n_kv; ++j) {
       ok = mbar_wait_warp(&s_full[t * 2 + (j & 1)], (j >> 1) & 1, abort_flag);
@@ -594,7 +605,7 @@ tc_attention_fast_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
       const uint32_t t_s = lane_base + (uint32_t)(j & 1) * kKT + (uint32_t)hh * kHalf;
       int valid = N - j * kKT - hh * kHalf;            // columns of this half that are keys
       valid = valid < 0 ? 0 : (valid > kHalf ? kHalf : valid);
-      if (j == 0) {
+      if (!PRESCALED && j == 0) {
         // First tile: the maximum over its (existing) keys becomes the row's scaling maximum for good.
         // Both halves read their columns, trade their maxima through shared memory, and then form P
         // from the scores they still hold in registers.
@@ -609,7 +620,8 @@ tc_attention_fast_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         xchg_m[(t * kQT + row) * 2 + hh] = m;
         __syncwarp();
         if (lane == 0) mbar_arrive(my_pair);
-        if (!(ok = mbar_wait_warp(my_pair, 0, abort_flag))) break;
+        if (!(ok = mbar_wait_warp(my_pair, pair_phase, abort_flag))) break;
+        pair_phase ^= 1;
         m = fmaxf(xchg_m[(t * kQT + row) * 2], xchg_m[(t * kQT + row) * 2 + 1]);   // finite: column 0 always exists
         nm2 = make_float2(-m * c, -m * c);
         bs = fmaf(-m, cs, 0.5f);
@@ -632,9 +644,9 @@ tc_attention_fast_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         }
         l_half = acc.x + acc.y;
       } else if (valid == kHalf) {
-        l_half += half_tile<false>(t_s, valid, c2, nm2, cs, bs);
+        l_half += half_tile<false, PRESCALED>(t_s, valid, c2, nm2, cs, bs);
       } else {
-        l_half += half_tile<true>(t_s, valid, c2, nm2, cs, bs);
+        l_half += half_tile<true, PRESCALED>(t_s, valid, c2, nm2, cs, bs);
       }
       tmem_st_wait();
       tc_fence_before();
@@ -646,12 +658,13 @@ tc_attention_fast_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
       xchg_l[(t * kQT + row) * 2 + hh] = l_half;
       __syncwarp();
       if (lane == 0) mbar_arrive(my_pair);
-      ok = mbar_wait_warp(my_pair, 1, abort_flag);
+      ok = mbar_wait_warp(my_pair, pair_phase, abort_flag);
     }
     if (ok) {
       const float l_row = xchg_l[(t * kQT + row) * 2] + xchg_l[(t * kQT + row) * 2 + 1];
       const int qi = (qg * kQTiles + t) * kQT + row;
-      const bool bad = qi < n_q && !(l_row < kRowSumLimit);          // also catches Inf and NaN
+      // (also catches Inf and NaN; without a maximum the sum must not be vanishingly small either)
+      const bool bad = qi < n_q && !(l_row < kRowSumLimit && (!PRESCALED || l_row > kRowSumFloor));
       if (__any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(cta_bad, 1);
       ok = mbar_wait_warp(&pv_full[t], 0, abort_flag);
       if (ok) {
@@ -717,7 +730,9 @@ static int attention_kernel_attributes() {
   return per_device_once(attr_once, [](int) {
     HERO_CUDA_TRY(cudaFuncSetAttribute(tc_attention_safe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)kAttSmem));
-    HERO_CUDA_TRY(cudaFuncSetAttribute(tc_attention_fast_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    HERO_CUDA_TRY(cudaFuncSetAttribute(tc_attention_fast_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)kFastSmem));
+    HERO_CUDA_TRY(cudaFuncSetAttribute(tc_attention_fast_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)kFastSmem));
     return HERO_OK;
   });
@@ -730,9 +745,11 @@ long long tc_attention_grid(int B, int n_q, int heads) {
 
 // d_status[0] counts CTAs that gave up; d_status[1 .. 1 + status_ctas) are the per-CTA words.  When the grid
 // fits in them the fast kernel runs, followed by the safe kernel on the CTAs the fast one marked; otherwise the
-// safe kernel does everything.
+// safe kernel does everything.  q_prescaled: the caller has multiplied Q by log2(e) / sqrt(head_dim) already, so
+// a score IS the exponent of its weight; the fast kernel then takes 2^s as it stands, with no maximum at all
+// (exact while a row's largest score stays within about +-100, the row sum telling when it did not).
 int launch_tc_attention(const void* q, const void* k, const void* v, void* o, int B, int n_q, int N, int heads,
-                        int* d_status, int status_ctas, cudaStream_t s) {
+                        bool q_prescaled, int* d_status, int status_ctas, cudaStream_t s) {
   if (B <= 0 || n_q <= 0) return HERO_OK;
   if (N <= 0 || heads <= 0) return HERO_ERR_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return HERO_ERR_ALIGN;
@@ -742,19 +759,24 @@ int launch_tc_attention(const void* q, const void* k, const void* v, void* o, in
   const long long grid = tc_attention_grid(B, n_q, heads);
   if (grid > 0x7FFFFFFFll) return HERO_ERR_ARG;
   int* cta_words = grid <= status_ctas ? d_status + 1 : nullptr;
-  if (cta_words)
-    tc_attention_fast_kernel<<<(unsigned)grid, kFastThreads, kFastSmem, s>>>(tm_q, tm_k, tm_v, (__nv_bfloat16*)o, n_q, N,
-                                                                             heads, d_status, cta_words);
-  tc_attention_safe_kernel<<<(unsigned)grid, kAttThreads, kAttSmem, s>>>(tm_q, tm_k, tm_v, (__nv_bfloat16*)o, n_q, N,
-                                                                         heads, d_status, cta_words);
+  if (cta_words) {
+    if (q_prescaled)
+      tc_attention_fast_kernel<true><<<(unsigned)grid, kFastThreads, kFastSmem, s>>>(
+          tm_q, tm_k, tm_v, (__nv_bfloat16*)o, n_q, N, heads, d_status, cta_words);
+    else
+      tc_attention_fast_kernel<false><<<(unsigned)grid, kFastThreads, kFastSmem, s>>>(
+          tm_q, tm_k, tm_v, (__nv_bfloat16*)o, n_q, N, heads, d_status, cta_words);
+  }
+  tc_attention_safe_kernel<<<(unsigned)grid, kAttThreads, kAttSmem, s>>>(
+      tm_q, tm_k, tm_v, (__nv_bfloat16*)o, n_q, N, heads, q_prescaled ? 1.0f : kScoreScaleLog2, d_status, cta_words);
   HERO_CUDA_TRY(cudaGetLastError());
   return HERO_OK;
 }
 
 // Test hook: the safe kernel alone on every CTA (what runs when there are no per-CTA words).
 int launch_tc_attention_safe(const void* q, const void* k, const void* v, void* o, int B, int n_q, int N, int heads,
-                             int* d_status, cudaStream_t s) {
-  return launch_tc_attention(q, k, v, o, B, n_q, N, heads, d_status, 0, s);
+                             bool q_prescaled, int* d_status, cudaStream_t s) {
+  return launch_tc_attention(q, k, v, o, B, n_q, N, heads, q_prescaled, d_status, 0, s);
 }
 
 }  // namespace hero
@@ -829,7 +851,7 @@ extern "C" int hero_attention_bf16_static(const void* d_q, const void* d_k, cons
   HERO_TRY(static_setup(&scratch));
   // the array still holds the previous call's records: clear the words this grid will use
   HERO_CUDA_TRY(cudaMemsetAsync(scratch, 0, (size_t)(1 + grid) * sizeof(int), s));
-  HERO_TRY(launch_tc_attention(d_q, d_k, d_v, d_o, B, n_q, N, heads, scratch, kStaticMaxCtas, s));
+  HERO_TRY(launch_tc_attention(d_q, d_k, d_v, d_o, B, n_q, N, heads, false, scratch, kStaticMaxCtas, s));
   if (h_gave_up) {
     HERO_CUDA_TRY(cudaMemcpyAsync(h_gave_up, scratch, sizeof(int), cudaMemcpyDeviceToHost, s));
     HERO_CUDA_TRY(cudaStreamSynchronize(s));

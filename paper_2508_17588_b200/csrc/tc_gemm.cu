@@ -225,6 +225,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
           const long long drow = out.scatter[seg] ? scat_row : (long long)m;
           __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(out.ptr[seg]) + drow * out.ld[seg] + col0;
           const float* gate = out.gate ? out.gate + (long long)b * out.gate_ld + col0 : nullptr;
+          const float seg_scale = (seg == 0 && out.seg0_scale != 0.f) ? out.seg0_scale : 1.0f;   // warp-uniform
 #pragma unroll
           for (int v = 0; v < 4; ++v) {        // 8 columns = one 16-byte store
             if (n0 + v * 8 < Nout) {
@@ -236,6 +237,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 float f0 = __uint_as_float(r[v * 8 + 2 * q]) + __uint_as_float(bw[q] << 16);
                 float f1 = __uint_as_float(r[v * 8 + 2 * q + 1]) + __uint_as_float(bw[q] & 0xFFFF0000u);
                 if (out.act == 1) { f0 = gelu_tanh_f(f0); f1 = gelu_tanh_f(f1); }
+                if (seg_scale != 1.0f) { f0 *= seg_scale; f1 *= seg_scale; }
                 if (gate) { f0 *= gate[v * 8 + 2 * q]; f1 *= gate[v * 8 + 2 * q + 1]; }
                 const __nv_bfloat162 p = __floats2bfloat162_rn(f0, f1);
                 packed[q] = *reinterpret_cast<const uint32_t*>(&p);

@@ -56,6 +56,16 @@ def test_gemm_many_tiles_per_cta():
 
 
 # ---------------------------------------------------------------- attention
+SCORE_SCALE_LOG2 = float(np.float32(0.125) * np.float32(1.4426950408889634))   # log2(e) / sqrt(64)
+
+
+def fold_softmax_scale(q):
+    """(what the q-scaled entry point is given, the queries that input stands for): q * log2(e)/8 rounded to
+    bf16, and that product divided by the factor again in float64."""
+    q_dev = S.round_bf16((q.astype(np.float64) * SCORE_SCALE_LOG2).astype(np.float32))
+    return q_dev, q_dev.astype(np.float64) / SCORE_SCALE_LOG2
+
+
 @pytest.mark.parametrize("B,n_q,N,heads", [(1, 128, 128, 1), (1, 1, 1, 1), (2, 37, 200, 2), (1, 130, 513, 3),
                                            (2, 300, 1000, 2), (1, 64, 2300, 1),
                                            # query counts around the 128-row tile and 256-row group edges: the
@@ -65,17 +75,21 @@ def test_gemm_many_tiles_per_cta():
                                            # key counts around the 96-key tile and the 48-column split of a row between
                                            # two threads: one half empty, one key in it, exactly one tile, one key more
                                            (1, 100, 48, 1), (2, 70, 49, 2), (1, 100, 96, 1), (3, 129, 95, 1), (1, 33, 145, 1)])
-@pytest.mark.parametrize("entry", ["hero_attention_bf16", "hero_attention_bf16_safe"])
+@pytest.mark.parametrize("entry", ["hero_attention_bf16", "hero_attention_bf16_safe", "hero_attention_bf16_q_scaled"])
 def test_attention_matches_oracle(B, n_q, N, heads, entry):
     rng = np.random.default_rng(B * 7 + n_q + N)
     D = heads * 64
     q = S.round_bf16(rng.standard_normal((B, n_q, D)).astype(np.float32))
+    if entry.endswith("q_scaled"):
+        q_dev, q = fold_softmax_scale(q)
+    else:
+        q_dev = q
     k = S.round_bf16(rng.standard_normal((B, N, D)).astype(np.float32))
     v = S.round_bf16(rng.standard_normal((B, N, D)).astype(np.float32))
     cfg = O.Config(n_blocks=1, n_shallow=1, hidden=D, n_heads=heads, head_dim=64, ffn_dim=8, temb_dim=8, batch=B,
                    frames=1, grid_h=1, grid_w=1, n_text=0, patch_h=1, patch_w=1, ratio_num=1, ratio_den=1)
     o = torch.full((B, n_q, D), float("nan"), device="cuda", dtype=torch.bfloat16)
-    getattr(H(), entry)(to_dev(q, "bf16"), to_dev(k, "bf16"), to_dev(v, "bf16"), o, heads)
+    getattr(H(), entry)(to_dev(q_dev, "bf16"), to_dev(k, "bf16"), to_dev(v, "bf16"), o, heads)
     H().hero_isolated_status()
     got = to_host(o)
     assert np.isfinite(got).all()
@@ -157,6 +171,44 @@ def test_attention_one_row_out_of_range_sends_only_its_thread_block_to_the_fallb
     for lo in (0, 256, 512):
         assert rel_l2(got[lo:lo + 256], want[lo:lo + 256]) <= 1e-2, lo
     assert np.abs(got[300] - v[0, 1234]).max() <= 2e-2             # that row returns the one key's value
+
+
+def test_q_scaled_attention_rows_outside_its_range_go_to_the_fallback():
+    """The q-scaled entry point takes 2^score with no row maximum, which holds while a row's largest score stays
+    within about +-100 (base-2 units).  Three thread blocks of queries: in the first every row is ordinary, in
+    the second one row's best key scores about +190, in the third one row's scores all lie near -220 (its sum of
+    weights underflows).  Both are recognised by their row sum and recomputed by the second kernel; every row of
+    every block must come out right."""
+    rng = np.random.default_rng(78)
+    n_q, N, D = 700, 1500, 64
+    q = rng.standard_normal((1, n_q, D)).astype(np.float32)
+    k = rng.standard_normal((1, N, D)).astype(np.float32)
+    v = rng.standard_normal((1, N, D)).astype(np.float32)
+    base = rng.standard_normal(D).astype(np.float32)
+    base /= np.linalg.norm(base)
+    u = q[0, 300] / np.linalg.norm(q[0, 300])
+    k[0, 1234] = 16.0 * u
+    k[0] += 12.0 * base                                             # every key has a common component
+    q[0, 300] = 64.0 * u                                            # q.k / 8 = 128 (natural units) at key 1234
+    q[0, 600] = -110.0 * base                                       # q.k / 8 ~ -150 for every key
+    q, k, v = S.round_bf16(q), S.round_bf16(k), S.round_bf16(v)
+    q_dev, q_eff = fold_softmax_scale(q)
+    s_log2 = np.einsum("qd,kd->qk", q_dev[0].astype(np.float64), k[0].astype(np.float64))
+    assert s_log2[300].max() > 150.0 and s_log2[600].max() < -150.0
+    others = np.delete(np.arange(n_q), [300, 600])
+    assert np.abs(s_log2[others]).max() < 60.0
+    cfg = O.Config(n_blocks=1, n_shallow=1, hidden=D, n_heads=1, head_dim=64, ffn_dim=8, temb_dim=8, batch=1,
+                   frames=1, grid_h=1, grid_w=1, n_text=0, patch_h=1, patch_w=1, ratio_num=1, ratio_den=1)
+    o = torch.full((1, n_q, D), float("nan"), device="cuda", dtype=torch.bfloat16)
+    H().hero_attention_bf16_q_scaled(to_dev(q_dev, "bf16"), to_dev(k, "bf16"), to_dev(v, "bf16"), o, 1)
+    H().hero_isolated_status()
+    got = to_host(o)[0]
+    assert np.isfinite(got).all()
+    want = O.attention(cfg, q_eff[0], k[0].astype(np.float64), v[0].astype(np.float64))
+    for lo in (0, 256, 512):
+        assert rel_l2(got[lo:lo + 256], want[lo:lo + 256]) <= 1e-2, lo
+    assert np.abs(got[300] - v[0, 1234]).max() <= 2e-2
+    assert np.abs(got[600] - want[600]).max() <= 3e-2 * np.abs(want[600]).max()
 
 
 # ---------------------------------------------------------------- bf16 blocks
