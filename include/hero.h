@@ -182,8 +182,8 @@ int hero_extrapolate_deep_stack(hero_ctx *ctx, void *d_x, int k, int d);
 int hero_step(hero_ctx *ctx, int step, void *d_x, const void *d_temb);
 /* Same with HOST buffers: copies h_x and h_temb to the device, runs the step, copies x
  * back into h_x and synchronises the stream.  With pinned (page-locked, device-visible) host buffers a cached
- * step overlaps both copies with the work: the first refresh block normalises its rows straight out of h_x
- * while x uploads on a second stream, and finished pieces of x travel back while the deep blocks run on the
+ * step overlaps both copies with the work: the first refresh block fetches its rows from h_x itself
+ * while x uploads on a second stream (the upload is awaited only by that block's residual pass), and finished pieces of x travel back while the deep blocks run on the
  * next piece.  Pageable buffers work too, without the overlap.  h_x must not be written by the caller during
  * the call. */
 int hero_step_host(hero_ctx *ctx, int step, void *h_x, const void *h_temb);

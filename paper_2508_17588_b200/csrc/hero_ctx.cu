@@ -37,7 +37,7 @@ constexpr unsigned kAllCaches = 0xFu;
 
 using namespace hero;
 
-constexpr int kHostPieces = 4;                 // pieces of x copied back while the next one is computed
+constexpr int kHostPieces = 8;                 // pieces of x copied back while the next one is computed
 constexpr long long kHostPieceAlign = 4096;    // elements; keeps every piece 16-byte aligned in both dtypes
 
 struct hero_ctx {
@@ -231,11 +231,22 @@ int refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, const i
   const float* gate2 = g.has_gate ? mod + 5 * D : nullptr;
 
   // attention branch
-  const void* x_rows = c->first_rows_src ? c->first_rows_src : d_x;
+  const void* host_rows = c->first_rows_src;
   c->first_rows_src = nullptr;
-  HERO_LAUNCH(c, HERO_PROF_GATHER_LN,
-              launch_gather_ln_modulate(x_rows, nullptr, d_idx, shift1, scale1, mod_ld, c->ws_a, B, N, n_sel, D, 1e-5f,
-                                        g.dtype, c->stream));
+  if (host_rows && d_idx) {
+    // x is still on its way to the device (hero_step_host): fetch the listed rows from the caller's pinned
+    // buffer, once, normalise them from that compact copy, and plant them in the device copy of x, where the
+    // FFN branch below will look for them.  The upload under way writes the same values over them.
+    HERO_LAUNCH(c, HERO_PROF_GATHER_LN, launch_gather_rows(host_rows, d_idx, c->ws_o, B, N, n_sel, D, g.dtype, c->stream));
+    HERO_LAUNCH(c, HERO_PROF_GATHER_LN,
+                launch_gather_ln_modulate(c->ws_o, nullptr, nullptr, shift1, scale1, mod_ld, c->ws_a, B, n_sel, n_sel, D,
+                                          1e-5f, g.dtype, c->stream));
+    HERO_LAUNCH(c, HERO_PROF_GATHER_LN, launch_scatter_rows(c->ws_o, d_idx, d_x, B, N, n_sel, D, g.dtype, c->stream));
+  } else {
+    HERO_LAUNCH(c, HERO_PROF_GATHER_LN,
+                launch_gather_ln_modulate(host_rows ? host_rows : d_x, nullptr, d_idx, shift1, scale1, mod_ld, c->ws_a, B,
+                                          N, n_sel, D, 1e-5f, g.dtype, c->stream));
+  }
   GemmOut o_qkv = {};
   o_qkv.ptr[0] = c->ws_q; o_qkv.ld[0] = D; o_qkv.scatter[0] = 0;
   o_qkv.ptr[1] = kdst;    o_qkv.ld[1] = D; o_qkv.scatter[1] = 1;
@@ -283,10 +294,6 @@ int refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, const i
   o_attn.gate = gate1; o_attn.gate_ld = mod_ld;
   HERO_TRY(run_gemm(c, c->ws_o, w.w_o, w.b_o, M, D, D, o_attn));
 
-  if (c->wait_x_upload) {                  // from here on x is read from the device copy
-    c->wait_x_upload = false;
-    HERO_CUDA_TRY(cudaStreamWaitEvent(c->stream, c->x_uploaded, 0));
-  }
   // FFN branch: its input rows are x + G_attn (the residual add is applied to x once, below)
   HERO_LAUNCH(c, HERO_PROF_GATHER_LN,
               launch_gather_ln_modulate(d_x, ga, d_idx, shift2, scale2, mod_ld, c->ws_a, B, N, n_sel, D, 1e-5f,
@@ -302,6 +309,10 @@ int refresh_block(hero_ctx* c, int block, void* d_x, const void* d_temb, const i
   HERO_TRY(run_gemm(c, c->ws_u, w.w_2, w.b_2, M, D, F, o_dn));
 
   // x = (x + G_attn) + G_ffn for every row: fresh rows and cached rows alike
+  if (c->wait_x_upload) {                  // every row of x is read from here on: the upload has to be complete
+    c->wait_x_upload = false;
+    HERO_CUDA_TRY(cudaStreamWaitEvent(c->stream, c->x_uploaded, 0));
+  }
   if (collapse) {
     HERO_LAUNCH(c, HERO_PROF_RESIDUAL,
                 launch_residual2_acc(d_x, ga, gf, c->stack_hist[c->stack_new], c->elems, g.dtype, c->stream));

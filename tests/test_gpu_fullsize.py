@@ -143,7 +143,7 @@ def test_grouped_deep_pass_full_size_sampled():
     deep blocks of the 42-block workload's cached step (56 history pairs streamed past x).  The histories are
     what two full passes leave on the device; every history tensor is read back once and sampled, the oracle
     applies Eq. 5 to the samples and adds them in block order.  Checked twice: through hero_step, and through
-    hero_step_host, which runs the pass over four row ranges and copies each back while the next is computed.
+    hero_step_host, which runs the pass over eight row ranges and copies each back while the next is computed.
     The real gap d = 3 and k = 2 are planted in the step record so that the slope is not the trivial one."""
     n_deep = 28
     cfgd = dict(S.CONFIGS["dit42"], n_blocks=n_deep, n_shallow=0, full_interval=0)
@@ -161,9 +161,9 @@ def test_grouped_deep_pass_full_size_sampled():
     k, d = 2, 3
     rng = np.random.default_rng(5)
     n_el = B * N * D
-    # sampled flat elements: random ones, the first and last packets, and the seams of the four-piece route
-    per = ((n_el + 3) // 4 + 4095) // 4096 * 4096                             # length of one piece
-    seams = np.concatenate([[p * per - 1, p * per] for p in range(1, 4)])
+    # sampled flat elements: random ones, the first and last packets, and the seams of the piece-by-piece route
+    per = ((n_el + 7) // 8 + 4095) // 4096 * 4096                             # length of one piece
+    seams = np.concatenate([[p * per - 1, p * per] for p in range(1, 8)])
     flat = np.unique(np.concatenate([rng.choice(n_el, 4000, replace=False), np.arange(16), n_el - 1 - np.arange(16), seams]))
     flat_t = torch.from_numpy(flat)
     pick = lambda t: t.reshape(-1)[flat_t].double().numpy()                  # sampled elements as float64
@@ -191,7 +191,7 @@ def test_grouped_deep_pass_full_size_sampled():
     h_x = x_before.cpu().pin_memory()
     hero.hero_step_host(5, h_x, temb.cpu().pin_memory())
     hero.hero_check_status()
-    assert torch.equal(h_x, x_a.cpu())                                      # the four-piece route: same bits
+    assert torch.equal(h_x, x_a.cpu())                                      # the piece-by-piece route: same bits
     hero.close()
 
     # The collapsed deep stack (deep_collapse = 1) at the same size and on the same inputs: its two fp32 sums must
