@@ -211,6 +211,40 @@ def test_q_scaled_attention_rows_outside_its_range_go_to_the_fallback():
     assert np.abs(got[600] - want[600]).max() <= 3e-2 * np.abs(want[600]).max()
 
 
+def test_q_scaled_attention_on_both_sides_of_its_range():
+    """Eight thread blocks of queries, each with its own level of scores: row maxima near +70, +90, +105, +120
+    and near -70, -88, -105, -118 (base-2 units; all keys of a row score between half the level and the level).
+    Levels inside +-100 are computed by the fast kernel as 2^score, the others are caught by their row sums
+    (beyond 2^100, below 2^-100) and recomputed by the second kernel; every block must match the oracle."""
+    rng = np.random.default_rng(5)
+    N, D = 300, 64
+    levels = [70.0, 90.0, 105.0, 120.0, -140.0, -180.0, -215.0, -240.0]      # alpha; maximum = alpha or alpha / 2
+    base = rng.standard_normal(D)
+    base /= np.linalg.norm(base)
+    beta = rng.uniform(0.5, 1.0, N)
+    beta[rng.integers(N)] = 1.0
+    k = S.round_bf16((beta[:, None] * base + 0.01 * rng.standard_normal((N, D)))[None].astype(np.float32))
+    v = S.round_bf16(rng.standard_normal((1, N, D)).astype(np.float32))
+    alpha = np.concatenate([lv + rng.uniform(-2.0, 2.0, 256) for lv in levels])
+    q_dev = S.round_bf16((alpha[:, None] * base)[None].astype(np.float32))   # already in exponent units
+    q_eff = q_dev.astype(np.float64) / SCORE_SCALE_LOG2
+    s_log2 = q_dev[0].astype(np.float64) @ k[0].astype(np.float64).T
+    top = s_log2.max(axis=1).reshape(len(levels), 256)
+    for c, want_top in enumerate([70, 90, 105, 120, -70, -88, -105, -118]):
+        assert np.abs(top[c] - want_top).max() < 5.0, (c, top[c].min(), top[c].max())
+    cfg = O.Config(n_blocks=1, n_shallow=1, hidden=D, n_heads=1, head_dim=64, ffn_dim=8, temb_dim=8, batch=1,
+                   frames=1, grid_h=1, grid_w=1, n_text=0, patch_h=1, patch_w=1, ratio_num=1, ratio_den=1)
+    o = torch.full((1, alpha.size, D), float("nan"), device="cuda", dtype=torch.bfloat16)
+    H().hero_attention_bf16_q_scaled(to_dev(q_dev, "bf16"), to_dev(k, "bf16"), to_dev(v, "bf16"), o, 1)
+    H().hero_isolated_status()
+    got = to_host(o)[0]
+    assert np.isfinite(got).all()
+    want = O.attention(cfg, q_eff[0], k[0].astype(np.float64), v[0].astype(np.float64))
+    for c in range(len(levels)):
+        sl = slice(256 * c, 256 * (c + 1))
+        assert rel_l2(got[sl], want[sl]) <= 1e-2, (c, rel_l2(got[sl], want[sl]))
+
+
 # ---------------------------------------------------------------- bf16 blocks
 SMALL_BF16 = dict(n_blocks=2, n_shallow=1, hidden=256, n_heads=4, head_dim=64, ffn_dim=768, temb_dim=64, batch=2,
                   frames=3, grid_h=9, grid_w=11, n_text=10, patch_h=2, patch_w=2, ratio_num=1, ratio_den=4,
