@@ -173,6 +173,43 @@ def test_attention_one_row_out_of_range_sends_only_its_thread_block_to_the_fallb
     assert np.abs(got[300] - v[0, 1234]).max() <= 2e-2             # that row returns the one key's value
 
 
+@pytest.mark.parametrize("entry", ["hero_attention_bf16", "hero_attention_bf16_q_scaled"])
+def test_fallback_serves_marked_thread_blocks_scattered_over_a_large_grid(entry):
+    """310 thread blocks of queries, more than two waves on the GPU's SMs; six of them, spread over the grid
+    (three of them 148 apart), hold one row that meets a key in the second key tile outscoring the rest by far
+    more than either fast kernel's range.  Exactly those blocks are recomputed by the fallback kernel; all 310
+    must match the oracle."""
+    rng = np.random.default_rng(91)
+    n_blocks, N, D = 310, 200, 64
+    n_q = n_blocks * 256
+    q = rng.standard_normal((1, n_q, D)).astype(np.float32)
+    k = rng.standard_normal((1, N, D)).astype(np.float32)
+    v = rng.standard_normal((1, N, D)).astype(np.float32)
+    u = k[0, 150] / np.linalg.norm(k[0, 150])
+    k[0, 150] = 16.0 * u
+    marked = [5, 7, 5 + 148, 200, 5 + 296, 309]
+    rows = [256 * c + 17 * (i + 1) for i, c in enumerate(marked)]
+    for r in rows:
+        q[0, r] = 128.0 * u                                        # q.k / 8 = 256 at key 150
+    q, k, v = S.round_bf16(q), S.round_bf16(k), S.round_bf16(v)
+    if entry.endswith("q_scaled"):
+        q_dev, q_eff = fold_softmax_scale(q)
+    else:
+        q_dev, q_eff = q, q.astype(np.float64)
+    cfg = O.Config(n_blocks=1, n_shallow=1, hidden=D, n_heads=1, head_dim=64, ffn_dim=8, temb_dim=8, batch=1,
+                   frames=1, grid_h=1, grid_w=1, n_text=0, patch_h=1, patch_w=1, ratio_num=1, ratio_den=1)
+    o = torch.full((1, n_q, D), float("nan"), device="cuda", dtype=torch.bfloat16)
+    getattr(H(), entry)(to_dev(q_dev, "bf16"), to_dev(k, "bf16"), to_dev(v, "bf16"), o, 1)
+    H().hero_isolated_status()
+    got = to_host(o)[0]
+    assert np.isfinite(got).all()
+    want = O.attention(cfg, q_eff[0], k[0].astype(np.float64), v[0].astype(np.float64))
+    err = np.array([rel_l2(got[256 * c:256 * (c + 1)], want[256 * c:256 * (c + 1)]) for c in range(n_blocks)])
+    assert err.max() <= 1e-2, (int(err.argmax()), float(err.max()))
+    for r in rows:
+        assert np.abs(got[r] - v[0, 150]).max() <= 2e-2, r
+
+
 def test_q_scaled_attention_rows_outside_its_range_go_to_the_fallback():
     """The q-scaled entry point takes 2^score with no row maximum, which holds while a row's largest score stays
     within about +-100 (base-2 units).  Three thread blocks of queries: in the first every row is ordinary, in
