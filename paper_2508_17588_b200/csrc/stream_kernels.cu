@@ -361,100 +361,94 @@ __global__ void __launch_bounds__(256) move_rows_kernel(const uint4* __restrict_
 }
 
 // ------------------------------------------------------------------ adaLN modulation vectors
-// mod[b, j] = b_mod[j] + sum_e silu(temb[b, e]) * w_mod[j, e]; one warp per output column j,
-// the weight row is read once with 16-byte loads and reused for every batch item.
-constexpr int kModMaxB = 8;
+// mod[b, j] = b_mod[j] + sum_e silu(temb[b, e]) * w_mod[j, e].  A warp owns kModRows consecutive output columns
+// j at a time: their weight rows are read once with 16-byte loads, all kModRows loads of a step in flight
+// together (a row of 512 weights is two loads per lane: one row at a time leaves the warp waiting on DRAM
+// latency for most of its life), and reused for every batch item.
+constexpr int kModMaxB = 8, kModRows = 4;
+
+// silu(temb) into shared memory, laid out [B][V::N][E / V::N]: element e of a row sits at
+// (e % V::N) * (E / V::N) + e / V::N, so that the lanes of a warp, which hold consecutive 16-byte packets of a
+// weight row, read consecutive words
 template <typename T>
-__global__ void __launch_bounds__(256) modulation_kernel(const T* __restrict__ temb, const T* __restrict__ w_mod,
-                                                         const T* __restrict__ b_mod, float* __restrict__ mod,
-                                                         int B, int n_out, int E) {
-  // silu(temb), laid out [B][V::N][E / V::N]: element e of a row sits at (e % V::N) * (E / V::N) + e / V::N, so
-  // that the lanes of a warp, which hold consecutive 16-byte packets of a weight row, read consecutive words
-  extern __shared__ float s_act[];
+__device__ __forceinline__ void modulation_stage_activations(const T* __restrict__ temb, float* s_act, int B, int E) {
   for (int i = threadIdx.x; i < B * E; i += blockDim.x) {
     const float t = to_f(temb[i]);
     const int b = i / E, e = i - b * E;
     s_act[b * E + (e % Vec<T>::N) * (E / Vec<T>::N) + e / Vec<T>::N] = t / (1.0f + expf(-t));
   }
   __syncthreads();
-  const int lane = threadIdx.x & 31;
-  const int warps_per_block = blockDim.x >> 5;
+}
+
+template <typename T, int MAXB>
+__device__ __forceinline__ void modulation_rows(const float* s_act, const T* __restrict__ w_mod,
+                                                const T* __restrict__ b_mod, float* __restrict__ mod, int B,
+                                                int n_out, int E) {
   using V = Vec<T>;
-  for (int j = blockIdx.x * warps_per_block + (threadIdx.x >> 5); j < n_out; j += gridDim.x * warps_per_block) {
-    float acc[kModMaxB];
+  const int lane = threadIdx.x & 31;
+  const int warps = gridDim.x * (blockDim.x >> 5), warp = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int packets = E / V::N;
+  for (int j0 = warp * kModRows; j0 < n_out; j0 += warps * kModRows) {
+    float acc[kModRows][MAXB];
 #pragma unroll
-    for (int b = 0; b < kModMaxB; ++b) acc[b] = 0.f;
-    const V* wrow = reinterpret_cast<const V*>(w_mod + (long long)j * E);
-    for (int c = lane; c < E / V::N; c += 32) {
-      float wf[V::N];
-      V wv; wv.raw = __ldg(&wrow[c].raw);
-      wv.unpack(wf);
+    for (int r = 0; r < kModRows; ++r)
 #pragma unroll
-      for (int b = 0; b < kModMaxB; ++b) {
+      for (int b = 0; b < MAXB; ++b) acc[r][b] = 0.f;
+#pragma unroll(MAXB <= 2 ? 2 : 1)
+    for (int c = lane; c < packets; c += 32) {
+      V wv[kModRows];
+#pragma unroll
+      for (int r = 0; r < kModRows; ++r) {
+        const int j = j0 + r < n_out ? j0 + r : n_out - 1;           // a row past the end repeats the last one
+        wv[r].raw = __ldg(&reinterpret_cast<const V*>(w_mod + (long long)j * E)[c].raw);
+      }
+      float wf[kModRows][V::N];
+#pragma unroll
+      for (int r = 0; r < kModRows; ++r) wv[r].unpack(wf[r]);
+#pragma unroll
+      for (int b = 0; b < MAXB; ++b) {
         if (b < B) {
 #pragma unroll
-          for (int q = 0; q < V::N; ++q) acc[b] = fmaf(s_act[b * E + q * (E / V::N) + c], wf[q], acc[b]);
+          for (int q = 0; q < V::N; ++q) {
+            const float a = s_act[b * E + q * packets + c];
+#pragma unroll
+            for (int r = 0; r < kModRows; ++r) acc[r][b] = fmaf(a, wf[r][q], acc[r][b]);
+          }
         }
       }
     }
 #pragma unroll
-    for (int b = 0; b < kModMaxB; ++b) {
-      if (b < B) {
-        float v = acc[b];
+    for (int r = 0; r < kModRows; ++r) {
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-        if (lane == 0) mod[(long long)b * n_out + j] = v + to_f(b_mod[j]);
+      for (int b = 0; b < MAXB; ++b) {
+        if (b < B) {
+          float v = acc[r][b];
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+          if (lane == 0 && j0 + r < n_out) mod[(long long)b * n_out + j0 + r] = v + to_f(b_mod[j0 + r]);
+        }
       }
     }
   }
 }
 
-// The same for several blocks at once: blockIdx.y picks the block's weights and output.
-template <typename T>
-__global__ void __launch_bounds__(256) modulation_batch_kernel(const T* __restrict__ temb, const ModBatch batch, int B,
-                                                               int n_out, int E) {
-  // silu(temb), laid out [B][V::N][E / V::N]: element e of a row sits at (e % V::N) * (E / V::N) + e / V::N, so
-  // that the lanes of a warp, which hold consecutive 16-byte packets of a weight row, read consecutive words
+template <typename T, int MAXB>
+__global__ void __launch_bounds__(256, 2) modulation_kernel(const T* __restrict__ temb, const T* __restrict__ w_mod,
+                                                         const T* __restrict__ b_mod, float* __restrict__ mod,
+                                                         int B, int n_out, int E) {
   extern __shared__ float s_act[];
-  for (int i = threadIdx.x; i < B * E; i += blockDim.x) {
-    const float t = to_f(temb[i]);
-    const int b = i / E, e = i - b * E;
-    s_act[b * E + (e % Vec<T>::N) * (E / Vec<T>::N) + e / Vec<T>::N] = t / (1.0f + expf(-t));
-  }
-  __syncthreads();
-  const T* __restrict__ w_mod = static_cast<const T*>(batch.w_mod[blockIdx.y]);
-  const T* __restrict__ b_mod = static_cast<const T*>(batch.b_mod[blockIdx.y]);
-  float* __restrict__ mod = batch.mod[blockIdx.y];
-  const int lane = threadIdx.x & 31;
-  const int warps_per_block = blockDim.x >> 5;
-  using V = Vec<T>;
-  for (int j = blockIdx.x * warps_per_block + (threadIdx.x >> 5); j < n_out; j += gridDim.x * warps_per_block) {
-    float acc[kModMaxB];
-#pragma unroll
-    for (int b = 0; b < kModMaxB; ++b) acc[b] = 0.f;
-    const V* wrow = reinterpret_cast<const V*>(w_mod + (long long)j * E);
-    for (int c = lane; c < E / V::N; c += 32) {
-      float wf[V::N];
-      V wv; wv.raw = __ldg(&wrow[c].raw);
-      wv.unpack(wf);
-#pragma unroll
-      for (int b = 0; b < kModMaxB; ++b) {
-        if (b < B) {
-#pragma unroll
-          for (int q = 0; q < V::N; ++q) acc[b] = fmaf(s_act[b * E + q * (E / V::N) + c], wf[q], acc[b]);
-        }
-      }
-    }
-#pragma unroll
-    for (int b = 0; b < kModMaxB; ++b) {
-      if (b < B) {
-        float v = acc[b];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-        if (lane == 0) mod[(long long)b * n_out + j] = v + to_f(b_mod[j]);
-      }
-    }
-  }
+  modulation_stage_activations<T>(temb, s_act, B, E);
+  modulation_rows<T, MAXB>(s_act, w_mod, b_mod, mod, B, n_out, E);
+}
+
+// The same for several blocks at once: blockIdx.y picks the block's weights and output.
+template <typename T, int MAXB>
+__global__ void __launch_bounds__(256, 2) modulation_batch_kernel(const T* __restrict__ temb, const ModBatch batch, int B,
+                                                               int n_out, int E) {
+  extern __shared__ float s_act[];
+  modulation_stage_activations<T>(temb, s_act, B, E);
+  modulation_rows<T, MAXB>(s_act, static_cast<const T*>(batch.w_mod[blockIdx.y]), static_cast<const T*>(batch.b_mod[blockIdx.y]),
+                     batch.mod[blockIdx.y], B, n_out, E);
 }
 
 // ------------------------------------------------------------------ gather + LayerNorm + modulate (Eq. 2 prologue)
@@ -759,21 +753,40 @@ int launch_scatter_rows(const void* src, const int* idx, void* dst, int B, int N
   return move_rows(false, src, idx, dst, B, N, n_sel, D, dtype, s);
 }
 
+// The kernels are instantiated for 1, 2, 4 and 8 batch items so that a warp's accumulators are as many as it needs.
+template <typename T, int MAXB>
+static void modulation_batch_launch(const void* temb, const ModBatch& batch, int B, int n_out, int E, dim3 grid,
+                                    size_t smem, cudaStream_t s) {
+  modulation_batch_kernel<T, MAXB><<<grid, 256, smem, s>>>((const T*)temb, batch, B, n_out, E);
+}
+template <typename T, int MAXB>
+static void modulation_launch(const void* temb, const void* w_mod, const void* b_mod, float* mod, int B, int n_out,
+                              int E, int blocks, size_t smem, cudaStream_t s) {
+  modulation_kernel<T, MAXB><<<blocks, 256, smem, s>>>((const T*)temb, (const T*)w_mod, (const T*)b_mod, mod, B, n_out, E);
+}
+#define HERO_MOD_DISPATCH(FN, T, ...)                      \
+  do {                                                     \
+    if (B <= 1) FN<T, 1>(__VA_ARGS__);                     \
+    else if (B <= 2) FN<T, 2>(__VA_ARGS__);                \
+    else if (B <= 4) FN<T, 4>(__VA_ARGS__);                \
+    else FN<T, kModMaxB>(__VA_ARGS__);                     \
+  } while (0)
+
 int launch_modulation_batch(const void* temb, const ModBatch& batch, int B, int n_out, int E, int dtype,
                             cudaStream_t s) {
   if (B > kModMaxB || batch.n < 0 || batch.n > kMaxModBatch) return HERO_ERR_ARG;
   if (batch.n == 0) return HERO_OK;
   const size_t smem = (size_t)B * E * sizeof(float);
-  int bx = (n_out + 7) / 8;
-  const int cap = num_sms() * 8 / batch.n;     // at most eight CTAs per SM over the whole grid: one wave, no tail
+  int bx = (n_out + 8 * kModRows - 1) / (8 * kModRows);     // eight warps per CTA, kModRows columns per warp and turn
+  const int cap = num_sms() * 2 / batch.n;     // two CTAs per SM over the whole grid (what the registers allow): one wave
   if (bx > cap) bx = cap < 1 ? 1 : cap;
   const dim3 grid(bx, batch.n);
   if (dtype == HERO_DTYPE_BF16) {
     if (E % 8) return HERO_ERR_ALIGN;
-    modulation_batch_kernel<__nv_bfloat16><<<grid, 256, smem, s>>>((const __nv_bfloat16*)temb, batch, B, n_out, E);
+    HERO_MOD_DISPATCH(modulation_batch_launch, __nv_bfloat16, temb, batch, B, n_out, E, grid, smem, s);
   } else {
     if (E % 4) return HERO_ERR_ALIGN;
-    modulation_batch_kernel<float><<<grid, 256, smem, s>>>((const float*)temb, batch, B, n_out, E);
+    HERO_MOD_DISPATCH(modulation_batch_launch, float, temb, batch, B, n_out, E, grid, smem, s);
   }
   HERO_CUDA_TRY(cudaGetLastError());
   return HERO_OK;
@@ -783,22 +796,20 @@ int launch_modulation(const void* temb, const void* w_mod, const void* b_mod, fl
                       int dtype, cudaStream_t s) {
   if (B > kModMaxB) return HERO_ERR_ARG;
   const size_t smem = (size_t)B * E * sizeof(float);
-  int blocks = (n_out + 7) / 8;
-  const int cap = num_sms() * 8;
+  int blocks = (n_out + 8 * kModRows - 1) / (8 * kModRows);
+  const int cap = num_sms() * 2;
   if (blocks > cap) blocks = cap;
   if (dtype == HERO_DTYPE_BF16) {
     if (E % 8) return HERO_ERR_ALIGN;
-    modulation_kernel<__nv_bfloat16><<<blocks, 256, smem, s>>>((const __nv_bfloat16*)temb,
-                                                                (const __nv_bfloat16*)w_mod,
-                                                                (const __nv_bfloat16*)b_mod, mod, B, n_out, E);
+    HERO_MOD_DISPATCH(modulation_launch, __nv_bfloat16, temb, w_mod, b_mod, mod, B, n_out, E, blocks, smem, s);
   } else {
     if (E % 4) return HERO_ERR_ALIGN;
-    modulation_kernel<float><<<blocks, 256, smem, s>>>((const float*)temb, (const float*)w_mod,
-                                                       (const float*)b_mod, mod, B, n_out, E);
+    HERO_MOD_DISPATCH(modulation_launch, float, temb, w_mod, b_mod, mod, B, n_out, E, blocks, smem, s);
   }
   HERO_CUDA_TRY(cudaGetLastError());
   return HERO_OK;
 }
+#undef HERO_MOD_DISPATCH
 
 int launch_gather_ln_modulate(const void* x, const void* add, const int* idx, const float* shift,
                               const float* scale, int mod_ld, void* a, int B, int N, int n_sel, int D, float eps,
