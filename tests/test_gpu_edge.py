@@ -73,6 +73,15 @@ def test_batch_three_with_gates_fp32():
     hero.close()
 
 
+@pytest.mark.parametrize("batch", [5, 8])
+def test_larger_batches_fp32(batch):
+    """Batch sizes beyond the workloads' 1 and 2: the adaLN kernel is instantiated for up to 1, 2, 4 and 8 items
+    (8 is the most the library takes), and every other kernel derives its row and batch indices from B."""
+    cfgd = dict(S.CONFIGS["tiny"], batch=batch, frames=1, grid_h=6, grid_w=5, n_text=3, steps=4, seed=29 + batch)
+    _, hero, _ = _run_steps(cfgd, 4, FP32_TOL)
+    hero.close()
+
+
 def test_reset_reproduces_the_run_bit_for_bit_and_contexts_are_independent():
     cfgd = dict(S.CONFIGS["tiny"], steps=5)
     _, hero, first = _run_steps(cfgd, 5, FP32_TOL)
