@@ -288,14 +288,15 @@ SMALL_BF16 = dict(n_blocks=2, n_shallow=1, hidden=256, n_heads=4, head_dim=64, f
                   quota_mode=0, warmup_full_steps=2, full_interval=3, dtype="bf16", has_gate=0, seed=21, steps=6)
 
 
-@pytest.mark.parametrize("gate,attend_mode,qk", [(0, 0, 0), (1, 0, 0), (0, 1, 0), (1, 1, 0), (0, 0, 1), (1, 1, 1)])
-def test_bf16_small_model_steps_teacher_forced(gate, attend_mode, qk):
+@pytest.mark.parametrize("gate,attend_mode,qk,batch", [(0, 0, 0, 2), (1, 0, 0, 2), (0, 1, 0, 2), (1, 1, 0, 2), (0, 0, 1, 2),
+                                                       (1, 1, 1, 2), (0, 0, 0, 1), (1, 0, 1, 3), (0, 1, 0, 5)])
+def test_bf16_small_model_steps_teacher_forced(gate, attend_mode, qk, batch):
     """Full, refresh and extrapolate blocks in bf16 over 6 steps (full at 0, 1, 4).  Each step both
     sides start from the same input; the oracle's caches are overwritten with the GPU's
     bf16 caches after every step (teacher forcing) so the per-step error is what is graded.
     attend_mode 1 restricts the keys of a cached step to the refreshed and text rows; qk = 1 turns on the
-    per-head LayerNorm and the rotary embedding of q and k."""
-    cfgd = dict(SMALL_BF16, has_gate=gate, attend_mode=attend_mode, qk_norm=qk, rope=qk)
+    per-head LayerNorm and the rotary embedding of q and k; batch sizes 1, 3 and 5 beside the workloads' 2."""
+    cfgd = dict(SMALL_BF16, has_gate=gate, attend_mode=attend_mode, qk_norm=qk, rope=qk, batch=batch)
     weights = [S.block_weights(cfgd, l) for l in range(cfgd["n_blocks"])]
     for w in weights:        # larger modulation so that scale/shift/gate matter
         w["w_mod"] = S.round_bf16(w["w_mod"] * 10)
