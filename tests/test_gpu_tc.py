@@ -296,7 +296,24 @@ def test_bf16_small_model_steps_teacher_forced(gate, attend_mode, qk, batch):
     bf16 caches after every step (teacher forcing) so the per-step error is what is graded.
     attend_mode 1 restricts the keys of a cached step to the refreshed and text rows; qk = 1 turns on the
     per-head LayerNorm and the rotary embedding of q and k; batch sizes 1, 3 and 5 beside the workloads' 2."""
-    cfgd = dict(SMALL_BF16, has_gate=gate, attend_mode=attend_mode, qk_norm=qk, rope=qk, batch=batch)
+    _bf16_steps_teacher_forced(dict(SMALL_BF16, has_gate=gate, attend_mode=attend_mode, qk_norm=qk, rope=qk, batch=batch))
+
+
+@pytest.mark.parametrize("over", [
+    dict(n_text=0),                                                    # no text rows at all
+    dict(n_text=0, attend_mode=1),                                     # ... and the refreshed rows as the only keys
+    dict(patch_h=2, patch_w=3, quota_mode=1, ratio_num=1, ratio_den=5, full_interval=2),   # the paper's selection
+    dict(patch_h=1, patch_w=1, ratio_num=1, ratio_den=3),              # one-token patches: quota 0 or 1 per patch
+    dict(frames=1, grid_h=23, grid_w=13, n_text=1, ratio_num=1, ratio_den=2),              # one frame, odd grid
+    dict(ratio_num=1, ratio_den=1),                                    # every token refreshed in cached steps
+], ids=["no_text", "no_text_literal_eq3", "paper_selection", "unit_patches", "one_frame_odd_grid", "ratio_one"])
+def test_bf16_small_model_steps_other_geometries(over):
+    """The same graded quantities on other token geometries and selection settings."""
+    _bf16_steps_teacher_forced(dict(SMALL_BF16, **over))
+
+
+def _bf16_steps_teacher_forced(cfgd):
+    gate = cfgd.get("has_gate", 0)
     weights = [S.block_weights(cfgd, l) for l in range(cfgd["n_blocks"])]
     for w in weights:        # larger modulation so that scale/shift/gate matter
         w["w_mod"] = S.round_bf16(w["w_mod"] * 10)
