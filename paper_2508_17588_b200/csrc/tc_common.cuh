@@ -71,13 +71,14 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   return mbar_wait_slow(bar, parity, abort_flag, budget_ns);
 }
 // The same wait for a whole warp whose lanes all poll the same barrier.  The lanes are brought together
-// first (a barrier among the lanes, not a vote), so that every lane enters the poll loop in the same
-// instruction: one poll is then one warp-wide instruction with one answer, the fast path is uniform, and
-// the vote at the end of the slow path always finds all 32 lanes - no lane can have left through the fast
-// path while the others wait for it in the vote.
-__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                               uint64_t budget_ns = kWaitBudgetNs) {
-  __syncwarp();
+// first (a barrier among the lanes, not a vote), so that every lane polls in the same instruction: one poll is
+// then one warp-wide instruction with one answer.  Nearly every wait in the kernels finds its phase complete
+// at that first poll (the producers run ahead), so that case is all the inlined code does: poll, vote, return.
+// Everything else - more polls, the bounded slow wait, the closing vote - sits in a function of its own that
+// the whole warp enters together (the first vote's answer is uniform), so no lane can leave through a fast
+// path while the others wait for it in a vote.
+static __device__ __noinline__ bool mbar_wait_warp_more(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                         uint64_t budget_ns) {
   bool done = false;
   for (uint32_t it = 0; it < kWaitFastPolls && !done; ++it) done = mbar_try_wait(bar, parity);
   // a completed phase stays completed, so lanes that saw it early and lanes that saw it late agree once all
@@ -85,6 +86,12 @@ __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, v
   if (__all_sync(0xFFFFFFFFu, done)) return true;
   if (!done) done = mbar_wait_slow(bar, parity, abort_flag, budget_ns);
   return __all_sync(0xFFFFFFFFu, done);
+}
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                               uint64_t budget_ns = kWaitBudgetNs) {
+  __syncwarp();
+  if (__all_sync(0xFFFFFFFFu, mbar_try_wait(bar, parity))) return true;
+  return mbar_wait_warp_more(bar, parity, abort_flag, budget_ns);
 }
 
 // ---------------------------------------------------------------- TMA (no multicast anywhere)
