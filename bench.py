@@ -35,7 +35,7 @@ sys.path.insert(0, ROOT)
 from workloads import synthetic as S  # noqa: E402
 
 METRIC = "hero_cached_step_tokens_per_s"
-ATTENTION_TRAFFIC_RATIO = 1.001   # dram__bytes_read+write / algorithmic bytes of tc_attention_fast_kernel<1> (ncu, small case: 0.998-1.003)
+ATTENTION_TRAFFIC_RATIO = 1.002   # dram__bytes_read+write / algorithmic bytes of tc_attention_fast_kernel<1> (ncu, small case: 0.998-1.006)
 UNIT = "tokens/s"
 NOMINAL_BF16_TFLOPS = 2250.0      # dense bf16, the figure the 60 % target is stated against
 NOMINAL_HBM_GBS = 8000.0          # the figure the 70 % target is stated against
