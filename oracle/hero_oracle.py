@@ -294,6 +294,8 @@ def attention(cfg: Config, q, k_all, v_all):
     because this is the plain definition."""
     n, hd = q.shape[0], cfg.head_dim
     out = np.empty((n, cfg.hidden), F64)
+    if n == 0:                 # an empty S(z): no query, nothing to attend (numpy cannot reduce an empty axis)
+        return out
     for h in range(cfg.n_heads):
         sl = slice(h * hd, (h + 1) * hd)
         s = q[:, sl] @ k_all[:, sl].T / np.sqrt(hd)

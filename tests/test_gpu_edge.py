@@ -45,6 +45,20 @@ def test_selection_lists_that_are_sometimes_empty():
     hero.close()
 
 
+@pytest.mark.parametrize("dtype,tol", [("fp32", FP32_TOL), ("bf16", 3e-2)])
+def test_no_text_rows_literal_eq3_and_selections_that_are_mostly_empty(dtype, tol):
+    """Two video tokens, no text rows, the refreshed rows as the only keys (attend_mode 1) and a ratio that
+    selects one token on some calls and none on most: cached steps whose refresh has neither queries nor keys."""
+    cfgd = dict(n_blocks=3, n_shallow=2, hidden=256, n_heads=4, head_dim=64, ffn_dim=128, temb_dim=64, batch=4,
+                frames=1, grid_h=1, grid_w=2, n_text=0, patch_h=3, patch_w=1, ratio_num=1, ratio_den=5, quota_mode=0,
+                warmup_full_steps=1, full_interval=0, dtype=dtype, has_gate=0, seed=1, steps=7, attend_mode=1)
+    cfg = O.Config.from_dict(cfgd)
+    lens = [O.n_selected(cfg, c) for c in range(6)]
+    assert 0 in lens and 1 in lens
+    _, hero, _ = _run_steps(cfgd, 7, tol)
+    hero.close()
+
+
 def test_ratio_one_refreshes_every_video_row_bf16():
     cfgd = dict(n_blocks=2, n_shallow=1, hidden=128, n_heads=2, head_dim=64, ffn_dim=256, temb_dim=64, batch=1,
                 frames=2, grid_h=5, grid_w=7, n_text=0, patch_h=2, patch_w=3, ratio_num=1, ratio_den=1,

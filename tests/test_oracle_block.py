@@ -322,6 +322,26 @@ def test_literal_eq3_attention_sees_only_refreshed_and_text_rows():
     np.testing.assert_allclose(st.g[0][bi, r], out @ orc.w[0]["w_o"].T + orc.w[0]["b_o"], rtol=1e-10, atol=1e-12)
 
 
+@pytest.mark.parametrize("attend_mode,n_text", [(0, 4), (1, 4), (1, 0)])
+def test_an_empty_selection_refreshes_nothing_and_adds_the_cached_outputs(attend_mode, n_text):
+    """S(z) empty (a quota of zero in every patch): Eq. 3 then keeps every cached row, no cache changes, and the
+    residual stream receives the cached branch outputs - also when the literal reading of Eq. 3 leaves the
+    refreshed queries no key at all (no text rows, no refreshed rows)."""
+    cfg = small_cfg(n_blocks=1, n_shallow=1, attend_mode=attend_mode, n_text=n_text)
+    w = rand_weights(cfg, seed=21)
+    rng = np.random.default_rng(22)
+    x0, temb0 = rng.standard_normal((2, cfg.n_rows, 32)), rng.standard_normal((2, 12))
+    x1, temb1 = rng.standard_normal((2, cfg.n_rows, 32)), rng.standard_normal((2, 12))
+    orc = O.HeroOracle(cfg, w)
+    orc.block_refresh(0, x0, temb0, None)
+    st = orc.blocks[0]
+    before = [a.copy() for a in (st.k_cache, st.v_cache, st.g[0], st.g[1])]
+    out = orc.block_refresh(0, x1.copy(), temb1, np.zeros(0, dtype=np.int64))
+    for a, b in zip((st.k_cache, st.v_cache, st.g[0], st.g[1]), before):
+        assert np.array_equal(a, b)
+    np.testing.assert_allclose(out, x1 + before[2] + before[3], rtol=1e-13, atol=1e-13)
+
+
 # ---------------------------------------------------------------- extrapolation (Eq. 5)
 def test_extrapolation_is_exact_on_features_linear_in_step():
     rng = np.random.default_rng(13)
